@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Benchmark of the SAGE decode-round hot path on B200.
+
+One step = one tree-verify round of the 16k-context video workload
+(configuration 4): fused entropy + top-10 over the draft logits [60 x 152064],
+entropy -> template for the next round (handed over on the device), tree-masked
+attention of the 60-node tree against a 16384-token paged bf16 cache for 80
+stacked layers, target argmax, greedy acceptance and KV compaction.
+
+  python bench.py --gpus N --steps K --warmup W            CUDA path (this repo)
+  python bench.py --impl reference --steps K --warmup W    the fp64 CPU oracle on the host cores
+
+Prints ONE JSON line.  With N > 1 (torchrun) every rank runs an independent
+replica of the round on its own GPU (the path has no exchange step); the time is
+the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import make_logits, make_target_logits, make_template, markov_entropy_states  # noqa: E402
+from workloads.gen import _rng  # noqa: E402
+
+CFG = 4
+HQ, HKV, D, P, V = 64, 8, 128, 64, 152064
+N_LAYERS, L_PREFIX, N_NODES, N_VISUAL = 80, 16384, 60, 32 * 196
+K_TOP, K_ENT, MAX_PATH, ROUNDS = 10, 10, 9, 8
+TEMPLATE_SHAPES = [(8, 2, N_NODES), (3, 10, N_NODES)]      # deep-narrow / shallow-wide, 60 nodes each
+THRESHOLDS = [0.5]
+WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefix (6272 visual + 10112 text), " \
+           "page 64 shuffled, 60-node tree, 80 layers, logits 60x152064 fp32"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def round_states():
+    for tid in range(5, 30):
+        states = markov_entropy_states(_rng(CFG, 50 + tid), ROUNDS, 0.8)
+        if len(set(states)) == 2:
+            return states
+    raise RuntimeError("no chain")
+
+
+def template_schedule(states, steps):
+    """Template used at step i: chosen from the confidence of the previous step's draft
+    logits (look-ahead); step 0 starts from alpha = 0.5 -> template 0."""
+    out = []
+    for i in range(steps):
+        out.append(0 if i == 0 else (0 if states[(i - 1) % ROUNDS] == 0 else 1))
+    return out
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [v.strip() for v in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 9] or [r for _, r in self.rows if len(r) >= 9]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[1]) for r in rows)
+        reasons = set()
+        for r in rows:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][2]), "reasons": sorted(reasons),
+                "samples": len(rows), "power_w_max": max(float(r[3]) for r in rows)}
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_seconds(rows_sample=6, heads_sample=1):
+    """Times the oracle, as it stands, on a bounded sample of one round: the logits side on
+    `rows_sample` of the 60 draft rows and as many target rows, attention of one layer for
+    `heads_sample` of the 8 KV heads, acceptance and compaction of one layer.  Returns the
+    seconds for that sample and the seconds of a full round extrapolated from it."""
+    import oracle
+    from workloads import make_kv_cache, make_q
+    tree = make_template(*TEMPLATE_SHAPES[1])
+    r = _rng(CFG, 900)
+    lg = make_logits(r, rows_sample, V, "high")["logits"]
+    kv = make_kv_cache(r, [L_PREFIX], [N_NODES], [N_VISUAL], heads_sample, shuffle=True, spare_frac=0.125)
+    G = HQ // HKV
+    q = make_q(r, N_NODES, heads_sample * G)[0]
+    offs = np.array([0, N_NODES], np.int32)
+    t0 = time.perf_counter()
+    _, lse = oracle.softmax_entropy(lg)
+    idx = oracle.topk(lg, K_TOP)
+    oracle.topk_logprob(lg, idx, lse)
+    _, alpha = oracle.confidence(lg, K_ENT)
+    oracle.select_tree(alpha[:1].astype(np.float32), THRESHOLDS)
+    oracle.topk(lg, 1)                                    # target argmax on as many rows
+    oracle.softmax_entropy(lg)
+    t_logits = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.tree_attention(q, kv["k_pool"][0], kv["v_pool"][0], kv["page_table"], kv["seq_len"], tree["parent"], offs,
+                          heads_sample * G, heads_sample, D, P, 1.0 / np.sqrt(D))
+    t_attn = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    rr = _rng(CFG, 901)
+    draft = rr.integers(0, 3, N_NODES).astype(np.int32)
+    target = rr.integers(0, 3, N_NODES).astype(np.int32)
+    path, plen, _ = oracle.accept(tree["parent"], draft, target, offs, MAX_PATH)
+    oracle.compact_kv(kv["k_pool"], kv["v_pool"], kv["page_table"], kv["seq_len"], path, plen, P)
+    t_tail = time.perf_counter() - t0
+    full = t_logits * (N_NODES / rows_sample) + t_attn * (HKV / heads_sample) * N_LAYERS \
+        + t_tail * (HKV / heads_sample) * N_LAYERS
+    return t_logits + t_attn + t_tail, full
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    for _ in range(args.warmup):
+        oracle_sample_seconds()
+    t0 = time.perf_counter()
+    fulls = []
+    for _ in range(args.steps):
+        _, full = oracle_sample_seconds()
+        fulls.append(full)
+    wall = time.perf_counter() - t0
+    full = float(np.mean(fulls))
+    value = 1.0 / full
+    sample = "per step: logits side on 6 of 60 rows (x10), attention + compaction of 1 of 8 KV heads of 1 of 80 " \
+             "layers (x640); a full round is extrapolated from the sample"
+    line = {"impl": "reference", "metric": "tree-verify rounds/s", "value": value, "unit": "rounds/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": full * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "n/a (CPU)"},
+            "cpu_baseline": {"value": value, "unit": "rounds/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "rounds/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "sample_wall_s": wall}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# CUDA path
+# ----------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2602_00523_b200 as sage
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(523000 + 1000 * CFG + 11 + rank)
+
+    # ---- resident state: paged K/V for 80 layers (generated on the device; perf-only data)
+    tot = L_PREFIX + N_NODES
+    used_pages = (tot + P - 1) // P
+    n_pages = int(np.ceil(used_pages * 1.125))
+    perm = _rng(CFG, 1).permutation(n_pages)[:used_pages]
+    page_table = torch.from_numpy(perm.astype(np.int32)).to(dev).view(1, -1)
+    k_pool = torch.empty((N_LAYERS, n_pages, HKV, P, D), dtype=torch.bfloat16, device=dev)
+    v_pool = torch.empty_like(k_pool)
+    vis_pages = torch.from_numpy(perm[:N_VISUAL // P].astype(np.int64)).to(dev)
+    for pool in (k_pool, v_pool):
+        for layer in range(N_LAYERS):
+            pool[layer].normal_(generator=gen)
+            pool[layer, vis_pages] *= 1.5
+    seq_len0 = torch.tensor([L_PREFIX], dtype=torch.int32, device=dev)
+    seq_len = seq_len0.clone()
+
+    # ---- templates and per-round inputs
+    tmpl = [make_template(*t) for t in TEMPLATE_SHAPES]
+    bank_p = np.full((2, 64), -1, np.int32)
+    bank_r = np.zeros((2, 64), np.int32)
+    for i, t in enumerate(tmpl):
+        bank_p[i, :N_NODES], bank_r[i, :N_NODES] = t["parent"], t["rank"]
+    bank_parent = torch.from_numpy(bank_p).to(dev)
+    bank_rank = torch.from_numpy(bank_r).to(dev)
+    bank_n = torch.tensor([N_NODES, N_NODES], dtype=torch.int32, device=dev)
+    policy = sage.make_policy(THRESHOLDS)
+    states = round_states()
+    total_steps = args.warmup + args.steps
+    sched = template_schedule(states, total_steps + 1)
+
+    node_offsets = torch.tensor([0, N_NODES], dtype=torch.int32, device=dev)
+    root_token = torch.tensor([int(_rng(CFG, 6).integers(0, V))], dtype=torch.int32, device=dev)
+    alpha_row = torch.zeros(1, dtype=torch.int32, device=dev)
+    status = sage.new_status(dev)
+
+    draft_host = [torch.from_numpy(make_logits(_rng(CFG, 100 + r), N_NODES, V, "low" if s == 0 else "high")["logits"])
+                  .pin_memory() for r, s in enumerate(states)]
+    draft_dev = [t.to(dev) for t in draft_host]
+    # target logits need the draft tokens of (round, template): one untimed expansion each
+    target_host, target_dev = {}, {}
+    for i in range(total_steps):
+        key = (i % ROUNDS, sched[i])
+        if key in target_host:
+            continue
+        t = tmpl[key[1]]
+        o = sage.sage_expand_topk(draft_dev[key[0]], K_TOP, K_ENT, parent=torch.from_numpy(t["parent"]).to(dev),
+                                  rank=torch.from_numpy(t["rank"]).to(dev), node_offsets=node_offsets,
+                                  root_token=root_token, status=status)
+        tok = o["draft_token"].cpu().numpy()
+        rr = _rng(CFG, 200 + key[0] * 2 + key[1])
+        leaf = int(rr.integers(N_NODES // 2, N_NODES))
+        tl = make_target_logits(rr, t, tok, leaf, V)["logits"]
+        target_host[key] = torch.from_numpy(tl).pin_memory()
+        target_dev[key] = target_host[key].to(dev)
+    q_host = torch.empty((N_LAYERS, N_NODES, HQ, D), dtype=torch.bfloat16).normal_().pin_memory()
+    q_dev = q_host.to(dev)
+    tree_kv_host = torch.empty((2, N_LAYERS, HKV, N_NODES, D), dtype=torch.bfloat16).normal_().pin_memory()
+    tree_page = int(perm[L_PREFIX // P])
+    assert L_PREFIX % P == 0 and N_NODES <= P
+
+    # ---- preallocated outputs / workspaces (no allocation inside the timed region)
+    ws_topk = torch.empty(sage.sage_expand_topk_workspace_size(N_NODES, V), dtype=torch.uint8, device=dev)
+    ws_attn = torch.empty(max(16, sage.sage_tree_attention_workspace_size(N_LAYERS, 1, N_NODES, HQ, HKV, D,
+                                                                          used_pages)), dtype=torch.uint8, device=dev)
+    out_draft, out_target, out_accept = {}, {}, {}
+    tree_buf = [{"next_parent": bank_parent[0].clone(), "next_rank": bank_rank[0].clone(),
+                 "next_node_offsets": node_offsets.clone()} for _ in range(2)]
+    sel_out = [dict(tb) for tb in tree_buf]
+    attn_out = torch.empty_like(q_dev)
+    result_host = torch.empty(MAX_PATH + 3, dtype=torch.int32).pin_memory()
+    result_dev = torch.empty(MAX_PATH + 3, dtype=torch.int32, device=dev)
+    attn_events = []
+
+    def one_round(i, from_host, time_attn):
+        r = i % ROUNDS
+        cur, nxt = tree_buf[i % 2], sel_out[(i + 1) % 2]
+        key = (r, sched[i])
+        if from_host:
+            draft = draft_in.copy_(draft_host[r], non_blocking=True)
+            target = target_in.copy_(target_host[key], non_blocking=True)
+            q = q_in.copy_(q_host, non_blocking=True)
+            k_pool[:, tree_page, :, :N_NODES, :].copy_(tree_kv_host[0], non_blocking=True)
+            v_pool[:, tree_page, :, :N_NODES, :].copy_(tree_kv_host[1], non_blocking=True)
+        else:
+            draft, target, q = draft_dev[r], target_dev[key], q_dev
+        d = sage.sage_expand_topk(draft, K_TOP, K_ENT, parent=cur["next_parent"], rank=cur["next_rank"],
+                                  node_offsets=node_offsets, root_token=root_token, out=out_draft, ws=ws_topk,
+                                  status=status)
+        sage.sage_select_tree(d["alpha"], policy, alpha_row=alpha_row, bank_parent=bank_parent, bank_rank=bank_rank,
+                              bank_n_nodes=bank_n, handover=True, out=nxt, status=status)
+        if time_attn:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        sage.sage_tree_attention(q, k_pool, v_pool, page_table, seq_len, cur["next_parent"], node_offsets,
+                                 1.0 / np.sqrt(D), out=attn_out, ws=ws_attn, status=status)
+        if time_attn:
+            e1.record()
+            attn_events.append((e0, e1))
+        t = sage.sage_expand_topk(target, 1, 1, out=out_target, ws=ws_topk, status=status)
+        a = sage.sage_accept(cur["next_parent"], d["draft_token"], t["topk_idx"], node_offsets, MAX_PATH,
+                             out=out_accept, status=status)
+        sage.sage_compact_kv(k_pool, v_pool, page_table, seq_len, a["path"], a["path_len"], status=status)
+        seq_len.copy_(seq_len0)                       # the next round starts from the same prefix length
+        if from_host:
+            result_dev[:MAX_PATH].copy_(a["path"][0])
+            result_dev[MAX_PATH:MAX_PATH + 1].copy_(a["path_len"])
+            result_dev[MAX_PATH + 1:MAX_PATH + 2].copy_(a["bonus_token"])
+            result_dev[MAX_PATH + 2:].copy_(nxt["template_id"])
+            result_host.copy_(result_dev, non_blocking=True)
+        return a, nxt
+
+    draft_in = torch.empty_like(draft_dev[0])
+    target_in = torch.empty_like(draft_dev[0])
+    q_in = torch.empty_like(q_dev)
+    # tree buffers alternate: sel_out[j] writes into tree_buf[j]'s tensors
+    for j in range(2):
+        sel_out[j]["template_id"] = torch.zeros(1, dtype=torch.int32, device=dev)
+        sel_out[j]["depth_cont"] = torch.zeros(1, dtype=torch.float32, device=dev)
+        sel_out[j]["width_cont"] = torch.zeros(1, dtype=torch.float32, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(from_host):
+        attn_events.clear()
+        for j in range(2):                            # both tree buffers restart from template 0
+            tree_buf[j]["next_parent"].copy_(bank_parent[0])
+            tree_buf[j]["next_rank"].copy_(bank_rank[0])
+        seen = []
+        for i in range(args.warmup):
+            one_round(i, from_host, False)
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        time.sleep(0.25)
+        t0 = time.time()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.warmup, total_steps):
+            _, nxt = one_round(i, from_host, True)
+            if from_host:
+                torch.cuda.current_stream().synchronize()     # the host consumes the result every step
+                seen.append(int(result_host[MAX_PATH + 2]))
+        e1.record()
+        barrier()
+        t1 = time.time()
+        clocks = sampler.stop(t0, t1)
+        ms = e0.elapsed_time(e1)
+        attn_ms = float(np.mean([a.elapsed_time(b) for a, b in attn_events]))
+        if world > 1:
+            tt = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        return ms, attn_ms, clocks, seen
+
+    ms, attn_ms, clocks, _ = timed(False)
+    if int(status.item()) != 0:
+        raise RuntimeError("device status: " + sage.status_string(int(status.item())))
+    e2e_ms, _, _, seen = timed(True)
+    expect = [sched[i + 1] for i in range(args.warmup, total_steps)]
+    if seen != expect:
+        raise RuntimeError(f"template sequence {seen} differs from the schedule {expect}")
+    if int(status.item()) != 0:
+        raise RuntimeError("device status: " + sage.status_string(int(status.item())))
+
+    if rank == 0:
+        steps = args.steps
+        value = world * steps / (ms * 1e-3)
+        e2e_value = world * steps / (e2e_ms * 1e-3)
+        M = N_NODES * (HQ // HKV)
+        flops = 4.0 * M * tot * D * HKV * N_LAYERS
+        kv_bytes = 2.0 * tot * HKV * D * 2 * N_LAYERS + 2.0 * N_NODES * HQ * D * 2 * N_LAYERS
+        ach_tf = flops / (attn_ms * 1e-3) / 1e12
+        ach_gb = kv_bytes / (attn_ms * 1e-3) / 1e9
+        h2d = draft_host[0].numel() * 4 * 2 + q_host.numel() * 2 + tree_kv_host.numel() * 2
+        sample_s, full_s = oracle_sample_seconds(rows_sample=N_NODES, heads_sample=HKV)
+        n_splits_gt1 = sage.sage_tree_attention_workspace_size(N_LAYERS, 1, N_NODES, HQ, HKV, D, used_pages) > 16
+        launches = 3 + 2 + (2 if n_splits_gt1 else 1) + 2 + 1 + 2
+        line = {
+            "metric": "tree-verify rounds/s", "value": value, "unit": "rounds/s", "n_gpus": world, "steps": steps,
+            "warmup": args.warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2: 5.4 GB of K/V streamed per step"},
+            "e2e": {"value": e2e_value, "unit": "rounds/s", "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(result_host.numel() * 4), "ms_per_step": e2e_ms / steps},
+            "gpu_launches": launches * steps,
+            "clocks": clocks,
+            "roofline": {"kernel": "tree_attention (80 stacked layers per launch)", "bound": "tensor",
+                         "achieved": ach_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": ach_tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                         "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
+                         "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": ach_gb / peaks["hbm_gbs"]}},
+            "cpu_baseline": {"value": 1.0 / full_s, "unit": "rounds/s", "cores": len(os.sched_getaffinity(0)),
+                             "kind": "oracle",
+                             "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
+                                       "rows), attention, acceptance and compaction of 1 of the 80 layers; the other "
+                                       "79 layers are extrapolated"},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

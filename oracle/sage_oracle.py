@@ -27,9 +27,10 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# Tree attention mask  (Section 2.2, "each token only attends to its
-# ancestors"; Algorithm 1, TreeAttnMask).  A node also sees itself: the chain
-# tree must reduce to ordinary causal attention, where a position sees itself.
+# Tree attention mask  (Section 2.2: the mask lets a tree token see its
+# ancestors only; Algorithm 1, TreeAttnMask).  A node also sees itself: the
+# chain tree must reduce to ordinary causal attention, where a position sees
+# itself.
 # --------------------------------------------------------------------------
 def ancestor_mask(parent: np.ndarray) -> np.ndarray:
     """anc[i] has bit j set iff j == i or j is an ancestor of i.  N <= 64."""
@@ -194,9 +195,10 @@ def expand_gather(topk_idx, parent, rank, node_offsets, root_token):
 
 
 # --------------------------------------------------------------------------
-# Greedy acceptance  (Section 2.2: "longest prefix matching the target's
-# predictions, advancing tau + 1 tokens"; Eq. 5; Section 3.3 "Phase 2": "all
-# draft tokens along the path match the corresponding greedy outputs").
+# Greedy acceptance  (Section 2.2: the acceptance length tau is that of the
+# longest prefix agreeing with the target's own predictions, and tau + 1 tokens
+# are committed; Eq. 5; Section 3.3 "Phase 2": every draft token on the chosen
+# path equals the target's greedy output at its parent).
 # --------------------------------------------------------------------------
 def accept(parent, draft_token, target_argmax, node_offsets, max_path):
     """Best path by enumeration of every root-to-leaf path.
@@ -244,8 +246,8 @@ def accept(parent, draft_token, target_argmax, node_offsets, max_path):
 
 
 # --------------------------------------------------------------------------
-# KV-cache update with the accepted tokens  (Algorithm 1, "Update KV caches
-# with accepted tokens"; Section 3.3 "Phase 2")
+# KV-cache update with the accepted tokens  (Algorithm 1, the cache-update
+# step that follows the acceptance step; Section 3.3 "Phase 2")
 # --------------------------------------------------------------------------
 def compact_kv(k_pool, v_pool, page_table, seq_len, path, path_len, page_size):
     """For every layer and KV head move the row at logical position

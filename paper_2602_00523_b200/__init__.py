@@ -1,0 +1,16 @@
+"""B200-native (sm_100a) kernels for the data-parallel hot path of a SAGE decode
+round: fused softmax-entropy + top-k, entropy -> tree template, tree-masked
+verification attention over a paged bf16 KV cache, greedy acceptance and KV
+compaction.  The product is the C-ABI library ``libsage.so`` (include/sage.h);
+this package is its thin ctypes binding.  Build it with
+``python -m paper_2602_00523_b200.build``.
+"""
+from .binding import (  # noqa: F401
+    SageError, SagePolicy, make_policy, new_status, status_string, lib,
+    sage_expand_topk, sage_expand_topk_workspace_size, sage_select_tree,
+    sage_build_ancestor_mask, sage_tree_attention, sage_tree_attention_workspace_size,
+    sage_accept, sage_compact_kv,
+    SAGE_OK, SAGE_ERR_INVALID_ARG, SAGE_ERR_UNSUPPORTED, SAGE_ERR_WORKSPACE, SAGE_ERR_CUDA,
+    SAGE_STATUS_BAD_TREE, SAGE_STATUS_BAD_PAGE, SAGE_STATUS_TIMEOUT, SAGE_STATUS_BAD_PATH,
+    SAGE_MAX_NODES, SAGE_MAX_TOPK, SAGE_MAX_TEMPLATES,
+)

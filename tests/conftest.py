@@ -8,6 +8,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+from paper_2602_00523_b200.build import build as _build_lib  # noqa: E402
+
+_build_lib()          # (re)compile libsage.so in-tree when a source is newer than the library
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200, sm_100a)")
 

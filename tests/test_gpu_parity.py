@@ -1,0 +1,401 @@
+"""GPU parity: every C-ABI entry point against the fp64 CPU oracle, element by
+element, on the same seeded inputs.  Bit-exact for indices, templates, paths and
+compacted caches; attention within max-abs 1e-2 and row-relative 1e-2; entropies
+within 1e-5 absolute."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2602_00523_b200 as sage
+from helpers import (ENTROPY_ABS, check_attention, dev_bf16, dev_f32, dev_i32, host_bits, oracle_attention_layer,
+                     oracle_logits_side, target_logits_for)
+from workloads import (TEMPLATES, bf16_bits, chain_tree, make_config, make_kv_cache, make_q, make_template,
+                       random_tree, star_tree)
+
+pytestmark = pytest.mark.gpu
+
+
+def rng(seed):
+    return np.random.Generator(np.random.Philox(seed))
+
+
+def gpu_attention(c, layers=None, status=None):
+    sl = slice(None) if layers is None else layers
+    q = dev_bf16(c["q"][sl])
+    k = dev_bf16(c["k_pool"][sl])
+    v = dev_bf16(c["v_pool"][sl])
+    st = status if status is not None else sage.new_status()
+    out = sage.sage_tree_attention(q, k, v, dev_i32(c["page_table"]), dev_i32(c["seq_len"]), dev_i32(c["parent"]),
+                                   dev_i32(c["node_offsets"]), c["sm_scale"], status=st)
+    torch.cuda.synchronize()
+    if status is None:
+        assert int(st.item()) == 0, sage.status_string(int(st.item()))
+    return host_bits(out)
+
+
+def gpu_logits(c, logits, k=None, ke=None, with_tree=True):
+    st = sage.new_status()
+    kw = {}
+    if with_tree:
+        kw = dict(parent=dev_i32(c["parent"]), rank=dev_i32(c["rank"]), node_offsets=dev_i32(c["node_offsets"]),
+                  root_token=dev_i32(c["root_token"]))
+    o = sage.sage_expand_topk(dev_f32(logits), k or c["k"], ke or c["k_entropy"], status=st, **kw)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return {n: t.cpu().numpy() for n, t in o.items()}
+
+
+def check_logits(got, lg, k, ke):
+    H, lse = oracle.softmax_entropy(lg)
+    idx = oracle.topk(lg, k)
+    Ht, alpha = oracle.confidence(lg, ke)
+    np.testing.assert_array_equal(got["topk_idx"], idx)
+    assert np.abs(got["entropy_full"] - H).max() <= ENTROPY_ABS
+    assert np.abs(got["entropy_topk"] - Ht).max() <= ENTROPY_ABS
+    assert np.abs(got["alpha"] - alpha).max() <= ENTROPY_ABS
+    assert np.abs(got["lse"] - lse).max() <= 1e-5 * max(1.0, np.abs(lse).max())
+    lp = oracle.topk_logprob(lg, idx, lse)
+    assert np.abs(got["topk_logprob"] - lp).max() <= 1e-5 * max(1.0, np.abs(lp).max())
+
+
+# ------------------------------------------------------------------ ancestors
+def test_ancestor_mask_batch():
+    r = rng(1)
+    trees = [random_tree(r, n) for n in (1, 2, 17, 64, 33)] + [chain_tree(64), star_tree(64)]
+    parent = np.concatenate([t["parent"] for t in trees])
+    offs = np.concatenate([[0], np.cumsum([len(t["parent"]) for t in trees])]).astype(np.int32)
+    st = sage.new_status()
+    anc = sage.sage_build_ancestor_mask(dev_i32(parent), dev_i32(offs), status=st).cpu().numpy().view(np.uint64)
+    assert int(st.item()) == 0
+    want = np.concatenate([oracle.ancestor_mask(t["parent"]) for t in trees])
+    np.testing.assert_array_equal(anc, want)
+
+
+def test_ancestor_mask_reports_bad_tree():
+    parent = np.array([-1, 0, 3, 1], dtype=np.int32)          # node 2 points forward
+    st = sage.new_status()
+    sage.sage_build_ancestor_mask(dev_i32(parent), dev_i32([0, 4]), status=st)
+    assert int(st.item()) == sage.SAGE_STATUS_BAD_TREE
+
+
+# ------------------------------------------------------------------ logits side
+@pytest.mark.parametrize("cfg", [1, 2, 3, 5])
+def test_expand_topk_configs(cfg):
+    c = make_config(cfg, scale_down=16)      # the logits do not depend on scale_down
+    lg = c["draft_logits"][0]
+    got = gpu_logits(c, lg)
+    check_logits(got, lg, c["k"], c["k_entropy"])
+    want = oracle_logits_side(c)
+    np.testing.assert_array_equal(got["draft_token"], want["draft_token"])
+
+
+def test_expand_topk_config4_all_rounds():
+    c = make_config(4, n_layers=1, scale_down=64)
+    assert len(c["draft_logits"]) == 8 and len(set(c["states"])) == 2
+    for r, lg in enumerate(c["draft_logits"]):
+        got = gpu_logits(c, lg)
+        check_logits(got, lg, c["k"], c["k_entropy"])
+        a = float(got["alpha"][0])
+        assert abs(a - 0.5) > 1e-4                           # far from the template threshold
+        assert (a >= 0.5) == (c["states"][r] == 0)
+
+
+def test_expand_topk_target_argmax_is_top1():
+    c = make_config(2, scale_down=16)
+    lg = c["draft_logits"][0]
+    got = gpu_logits(c, lg, k=1, ke=1, with_tree=False)
+    np.testing.assert_array_equal(got["topk_idx"][:, 0], lg.astype(np.float64).argmax(axis=1))
+    np.testing.assert_array_equal(got["alpha"], np.ones(len(lg), np.float32))
+    np.testing.assert_array_equal(got["topk_idx"][:, 0], c["draft_peak"][0])
+
+
+@pytest.mark.parametrize("vocab,rows", [(17, 3), (1000, 5), (4099, 7), (32000, 15), (152064, 2), (8192 * 5 + 1, 300)])
+@pytest.mark.parametrize("k", [1, 4, 16])
+def test_expand_topk_shapes_and_ragged_vocab(vocab, rows, k):
+    r = rng(vocab + k)
+    stride = (vocab + 3) // 4 * 4 + 8                        # padded rows: stride != vocab
+    buf = r.standard_normal((rows, stride)).astype(np.float32) * 3
+    buf[:, vocab:] = 1e9                                     # padding must never be read
+    lg = buf[:, :vocab]
+    st = sage.new_status()
+    dbuf = dev_f32(buf)
+    o = sage.sage_expand_topk(dbuf[:, :vocab], k, min(k, 10), status=st)
+    got = {n: t.cpu().numpy() for n, t in o.items()}
+    check_logits(got, np.ascontiguousarray(lg), k, min(k, 10))
+
+
+def test_expand_topk_ties_constant_rows_and_signed_zero():
+    V = 152064
+    lg = np.zeros((6, V), np.float32)
+    lg[0, :] = 1.25                                          # constant row: indices 0..k-1, H = ln V
+    lg[1, :] = -3.0
+    lg[1, [5, 40000, 152063, 76032, 76031]] = 2.0            # five-way tie across chunk boundaries
+    lg[2] = rng(5).integers(-4, 5, V).astype(np.float32)     # massive ties everywhere
+    lg[3, :] = -1.0
+    lg[3, 100], lg[3, 50] = 0.0, -0.0                        # -0 == +0: lower index first
+    lg[4] = np.sort(rng(6).standard_normal(V).astype(np.float32))          # ascending: worst case for the queues
+    lg[5] = np.sort(rng(7).standard_normal(V).astype(np.float32))[::-1]    # descending
+    for k in (3, 10, 16):
+        got = gpu_logits(None, lg, k=k, ke=k, with_tree=False)
+        check_logits(got, lg, k, k)
+    got = gpu_logits(None, lg, k=4, ke=4, with_tree=False)
+    assert list(got["topk_idx"][0]) == [0, 1, 2, 3]
+    assert abs(got["entropy_full"][0] - np.log(V)) <= ENTROPY_ABS
+    assert list(got["topk_idx"][1]) == [5, 40000, 76031, 76032]
+    assert list(got["topk_idx"][3][:2]) == [50, 100]
+    assert abs(got["alpha"][0]) <= ENTROPY_ABS               # uniform top-k -> alpha = 0
+
+
+def test_expand_topk_one_hot_row_has_zero_entropy():
+    V = 152064
+    lg = np.zeros((2, V), np.float32)
+    lg[0, 777] = 1e4
+    lg[1, 3] = 60.0
+    got = gpu_logits(None, lg, k=10, ke=10, with_tree=False)
+    check_logits(got, lg, 10, 10)
+    assert abs(got["entropy_full"][0]) <= ENTROPY_ABS and got["alpha"][0] == 1.0
+
+
+def test_expand_topk_is_deterministic():
+    c = make_config(3, scale_down=16)
+    a = gpu_logits(c, c["draft_logits"][0])
+    b = gpu_logits(c, c["draft_logits"][0])
+    for n in a:
+        np.testing.assert_array_equal(a[n].view(np.int32), b[n].view(np.int32))
+
+
+# ------------------------------------------------------------------ selection
+def test_select_tree_matches_oracle_on_gpu_alphas():
+    c = make_config(5, scale_down=16)
+    got = gpu_logits(c, c["draft_logits"][0])
+    alpha = got["alpha"]                                     # the fp32 array both sides decide on
+    rows = c["node_offsets"][:-1]                            # root row of every sequence
+    thr = [0.8, 0.4, 0.1]
+    for t in thr:
+        assert np.abs(alpha[rows] - t).min() > 1e-4
+    pol = sage.make_policy(thr)
+    o = sage.sage_select_tree(dev_f32(alpha), pol, alpha_row=dev_i32(rows))
+    tid, D, W = oracle.select_tree(alpha[rows], thr)
+    np.testing.assert_array_equal(o["template_id"].cpu().numpy(), tid)
+    np.testing.assert_allclose(o["depth_cont"].cpu().numpy(), D, atol=1e-6)
+    np.testing.assert_allclose(o["width_cont"].cpu().numpy(), W, atol=1e-6)
+    assert sorted(set(tid.tolist())) == [0, 1, 2, 3]         # the config exercises all four templates
+    np.testing.assert_array_equal(tid, c["states"])          # and lands each sequence in its intended band
+
+
+def test_select_tree_edges_and_handover():
+    thr = [0.8, 0.4, 0.1]
+    a = np.float32([0.0, 1.0, 0.5, 0.8, np.nextafter(np.float32(0.8), np.float32(0)), 0.4, 0.1, 0.0999])
+    bank_p = np.full((4, 64), -1, np.int32)
+    bank_r = np.zeros((4, 64), np.int32)
+    bank_n = np.zeros(4, np.int32)
+    tmpl = [make_template(*t) for t in TEMPLATES]
+    for i, t in enumerate(tmpl):
+        n = len(t["parent"])
+        bank_p[i, :n], bank_r[i, :n], bank_n[i] = t["parent"], t["rank"], n
+    st = sage.new_status()
+    o = sage.sage_select_tree(dev_f32(a), sage.make_policy(thr), bank_parent=dev_i32(bank_p), bank_rank=dev_i32(bank_r),
+                              bank_n_nodes=dev_i32(bank_n), handover=True, status=st)
+    assert int(st.item()) == 0
+    tid, D, W = oracle.select_tree(a, thr)
+    np.testing.assert_array_equal(o["template_id"].cpu().numpy(), tid)
+    assert list(tid) == [3, 0, 1, 0, 1, 1, 2, 3]
+    got_D, got_W = o["depth_cont"].cpu().numpy(), o["width_cont"].cpu().numpy()
+    assert got_D[0] == 3 and got_D[1] == 8 and got_D[2] == 5.5 and got_W[0] == 10 and got_W[1] == 2 and got_W[2] == 6
+    offs = o["next_node_offsets"].cpu().numpy()
+    np.testing.assert_array_equal(offs, np.concatenate([[0], np.cumsum(bank_n[tid])]))
+    np_, nr_ = o["next_parent"].cpu().numpy(), o["next_rank"].cpu().numpy()
+    for b, t in enumerate(tid):
+        np.testing.assert_array_equal(np_[offs[b]:offs[b + 1]], tmpl[t]["parent"])
+        np.testing.assert_array_equal(nr_[offs[b]:offs[b + 1]], tmpl[t]["rank"])
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_tree_attention_configs(cfg):
+    c = make_config(cfg)
+    got = gpu_attention(c)
+    check_attention(got[0], oracle_attention_layer(c, 0))
+
+
+def test_tree_attention_config4_three_layers_full_context():
+    c = make_config(4, n_layers=3)                           # L = 16384, shuffled pages, 60 nodes
+    got = gpu_attention(c)                                   # stacked-layer launch
+    for layer in range(3):
+        check_attention(got[layer], oracle_attention_layer(c, layer))
+    one = gpu_attention(c, layers=slice(1, 2))               # single-layer launch takes the split-K path
+    check_attention(one[0], oracle_attention_layer(c, 1))
+
+
+def test_tree_attention_config5_ragged_batch():
+    c = make_config(5)
+    got = gpu_attention(c)
+    check_attention(got[0], oracle_attention_layer(c, 0))
+
+
+@pytest.mark.parametrize("L,N,G", [(0, 1, 8), (0, 64, 8), (1, 7, 4), (63, 2, 8), (64, 64, 8), (65, 33, 2),
+                                   (127, 60, 8), (200, 64, 1), (1000, 17, 8), (4097, 64, 8)])
+def test_tree_attention_edges(L, N, G):
+    r = rng(L * 100 + N)
+    Hkv = 2
+    tree = random_tree(r, N)
+    kv = make_kv_cache(r, [L], [N], [L // 2], Hkv, shuffle=True, spare_frac=0.3)
+    c = {"q": make_q(r, N, Hkv * G), **kv, "parent": tree["parent"], "node_offsets": np.array([0, N], np.int32),
+         "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.11}
+    got = gpu_attention(c)
+    check_attention(got[0], oracle_attention_layer(c, 0))
+
+
+def test_tree_attention_chain_and_star_trees():
+    r = rng(9)
+    for tree in (chain_tree(40), star_tree(50)):
+        N = len(tree["parent"])
+        kv = make_kv_cache(r, [300], [N], [100], 2)
+        c = {"q": make_q(r, N, 16), **kv, "parent": tree["parent"], "node_offsets": np.array([0, N], np.int32),
+             "n_q_heads": 16, "n_kv_heads": 2, "head_dim": 128, "page_size": 64, "sm_scale": 0.0884}
+        check_attention(gpu_attention(c)[0], oracle_attention_layer(c, 0))
+
+
+def test_tree_attention_reports_bad_page_and_bad_tree():
+    c = make_config(1)
+    bad = dict(c)
+    bad["page_table"] = c["page_table"].copy()
+    bad["page_table"][0, 1] = 10 ** 6
+    st = sage.new_status()
+    gpu_attention(bad, status=st)
+    assert int(st.item()) == sage.SAGE_STATUS_BAD_PAGE
+    bad = dict(c)
+    bad["parent"] = c["parent"].copy()
+    bad["parent"][5] = 9
+    st = sage.new_status()
+    gpu_attention(bad, status=st)
+    assert int(st.item()) == sage.SAGE_STATUS_BAD_TREE
+    bad = dict(c)
+    bad["seq_len"] = np.array([10 ** 6], np.int32)           # longer than the page table allows
+    st = sage.new_status()
+    gpu_attention(bad, status=st)
+    assert int(st.item()) == sage.SAGE_STATUS_BAD_PAGE
+
+
+def test_tree_attention_is_deterministic():
+    c = make_config(3, scale_down=4)
+    np.testing.assert_array_equal(gpu_attention(c), gpu_attention(c))
+
+
+# ------------------------------------------------------------------ acceptance
+def gpu_accept(parent, draft, target, offs, max_path):
+    st = sage.new_status()
+    o = sage.sage_accept(dev_i32(parent), dev_i32(draft), dev_i32(target), dev_i32(offs), max_path, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return o["path"].cpu().numpy(), o["path_len"].cpu().numpy(), o["bonus_token"].cpu().numpy()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_accept_random_batches(seed):
+    r = rng(500 + seed)
+    B = 37
+    trees = [random_tree(r, int(r.integers(1, 65))) for _ in range(B)]
+    parent = np.concatenate([t["parent"] for t in trees])
+    offs = np.concatenate([[0], np.cumsum([len(t["parent"]) for t in trees])]).astype(np.int32)
+    alphabet = 1 + seed % 3
+    draft = r.integers(0, alphabet, len(parent)).astype(np.int32)
+    target = r.integers(0, alphabet, len(parent)).astype(np.int32)
+    for max_path in (1, 4, 9, 64):
+        got = gpu_accept(parent, draft, target, offs, max_path)
+        want = oracle.accept(parent, draft, target, offs, max_path)
+        for g, w in zip(got, want):
+            np.testing.assert_array_equal(g, w)
+
+
+def test_accept_chain_of_64_and_templates():
+    t = chain_tree(64)
+    draft = np.arange(64, dtype=np.int32) + 100
+    target = np.arange(64, dtype=np.int32) + 101
+    offs = np.array([0, 64], np.int32)
+    path, plen, bonus = gpu_accept(t["parent"], draft, target, offs, 64)
+    assert plen[0] == 64 and bonus[0] == 164 and list(path[0]) == list(range(64))
+    for tm in TEMPLATES:
+        tr = make_template(*tm)
+        n = len(tr["parent"])
+        r = rng(n)
+        d = r.integers(0, 3, n).astype(np.int32)
+        tg = r.integers(0, 3, n).astype(np.int32)
+        got = gpu_accept(tr["parent"], d, tg, np.array([0, n], np.int32), 9)
+        want = oracle.accept(tr["parent"], d, tg, np.array([0, n], np.int32), 9)
+        for g, w in zip(got, want):
+            np.testing.assert_array_equal(g, w)
+
+
+# ------------------------------------------------------------------ compaction
+def run_compaction(kv, paths, plen, n_layers):
+    k, v = dev_bf16(kv["k_pool"]), dev_bf16(kv["v_pool"])
+    sl = dev_i32(kv["seq_len"])
+    st = sage.new_status()
+    sage.sage_compact_kv(k, v, dev_i32(kv["page_table"]), sl, dev_i32(paths), dev_i32(plen), status=st)
+    torch.cuda.synchronize()
+    return host_bits(k), host_bits(v), sl.cpu().numpy(), int(st.item())
+
+
+def test_compact_kv_whole_pool_bit_exact():
+    r = rng(77)
+    B, layers = 5, 3
+    L = [100, 64, 1, 700, 129]
+    N = [24, 60, 64, 36, 48]
+    kv = make_kv_cache(r, L, N, [50, 10, 0, 300, 64], 4, n_layers=layers, shuffle=True, spare_frac=0.25, poison=False)
+    kv["k_pool"] = r.integers(0, 65536, kv["k_pool"].shape).astype(np.uint16)      # arbitrary bytes, NaNs included
+    kv["v_pool"] = r.integers(0, 65536, kv["v_pool"].shape).astype(np.uint16)
+    paths = np.full((B, 9), -1, np.int32)
+    rows = [[0, 2, 3], [0], [0, 1, 2, 3, 4, 5, 6, 7, 63], [0, 5, 9, 20, 35], [0, 1, 2]]
+    for b, p in enumerate(rows):
+        paths[b, :len(p)] = p
+    plen = np.array([len(p) for p in rows], np.int32)
+    k2, v2, sl, st = run_compaction(kv, paths, plen, layers)
+    assert st == 0
+    wk, wv, wl = oracle.compact_kv(kv["k_pool"], kv["v_pool"], kv["page_table"], kv["seq_len"], paths, plen, 64)
+    np.testing.assert_array_equal(k2, wk)
+    np.testing.assert_array_equal(v2, wv)
+    np.testing.assert_array_equal(sl, wl)
+
+
+def test_compact_kv_rejects_bad_path_without_touching_the_pool():
+    r = rng(78)
+    kv = make_kv_cache(r, [100], [24], [50], 2, poison=False)
+    paths = np.array([[0, 5, 3, -1]], np.int32)               # not increasing
+    k2, v2, sl, st = run_compaction(kv, paths, np.array([3], np.int32), 1)
+    assert st == sage.SAGE_STATUS_BAD_PATH
+    np.testing.assert_array_equal(k2, kv["k_pool"])
+    np.testing.assert_array_equal(v2, kv["v_pool"])
+
+
+# ------------------------------------------------------------------ whole round
+@pytest.mark.parametrize("cfg", [1, 2, 3, 5])
+def test_full_round_against_oracle(cfg):
+    """expand -> select -> attention -> target argmax -> accept -> compact, GPU vs oracle."""
+    c = make_config(cfg, scale_down=1 if cfg == 1 else 8, n_layers=2)
+    want = oracle_logits_side(c)
+    got = gpu_logits(c, c["draft_logits"][0])
+    np.testing.assert_array_equal(got["topk_idx"], want["topk_idx"])
+    np.testing.assert_array_equal(got["draft_token"], want["draft_token"])
+    # target logits are built from the ORACLE's draft tokens
+    tl, _ = target_logits_for(c, want["draft_token"])
+    tgt = gpu_logits(c, tl, k=1, ke=1, with_tree=False)["topk_idx"][:, 0]
+    want_tgt = oracle.topk(tl, 1)[:, 0]
+    np.testing.assert_array_equal(tgt, want_tgt)
+    max_path = 9
+    g_path, g_len, g_bonus = gpu_accept(c["parent"], got["draft_token"], tgt, c["node_offsets"], max_path)
+    w_path, w_len, w_bonus = oracle.accept(c["parent"], want["draft_token"], want_tgt, c["node_offsets"], max_path)
+    np.testing.assert_array_equal(g_path, w_path)
+    np.testing.assert_array_equal(g_len, w_len)
+    np.testing.assert_array_equal(g_bonus, w_bonus)
+    assert w_len.max() > 1                                    # the planted path was found
+    out = gpu_attention(c)
+    for layer in range(2):
+        check_attention(out[layer], oracle_attention_layer(c, layer))
+    k2, v2, sl, st = run_compaction(c, g_path, g_len, 2)
+    assert st == 0
+    wk, wv, wl = oracle.compact_kv(c["k_pool"], c["v_pool"], c["page_table"], c["seq_len"], w_path, w_len, 64)
+    np.testing.assert_array_equal(k2, wk)
+    np.testing.assert_array_equal(v2, wv)
+    np.testing.assert_array_equal(sl, wl)

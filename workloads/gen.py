@@ -338,7 +338,11 @@ def make_config(cfg: int, n_layers: Optional[int] = None, rounds: Optional[int] 
         trees = [make_template(8, 2, N)]
         kv = make_kv_cache(_rng(cfg, 1), L, [N], nvis, Hkv, n_layers=n_layers or 3,
                            shuffle=True, spare_frac=0.125)
-        states = markov_entropy_states(_rng(cfg, 5), rounds or 8, 0.8)
+        # the first seeded chain (tensor ids 5, 6, ...) that visits both states
+        for tid in range(5, 30):
+            states = markov_entropy_states(_rng(cfg, 50 + tid), rounds or 8, 0.8)
+            if len(set(states)) == 2 or (rounds or 8) < 2:
+                break
         draft = [make_logits(_rng(cfg, 100 + r), N, V, "low" if s == 0 else "high")
                  for r, s in enumerate(states)]
     elif cfg == 5:
@@ -353,7 +357,7 @@ def make_config(cfg: int, n_layers: Optional[int] = None, rounds: Optional[int] 
         kv = make_kv_cache(_rng(cfg, 1), L, [len(t["parent"]) for t in trees], nvis, Hkv,
                            n_layers=n_layers or 1, shuffle=True, spare_frac=0.1)
         # planted margins that land alpha in the four bands (>=0.8, 0.4-0.8, 0.1-0.4, <0.1)
-        kinds_by_band = ["low", "mid:3.0", "mid:2.0", "high"]
+        kinds_by_band = ["low", "mid:3.0", "mid:1.8", "high"]
         rows = []
         for b in range(B):
             rows.extend([kinds_by_band[band[b]]] * len(trees[b]["parent"]))
