@@ -1,87 +1,192 @@
 // Tree-masked verification attention over a paged bf16 KV cache (Section 2.2;
-// Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2).
+// Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2), sm_100a.
 //
-// Flash-decoding layout: the N tree nodes x G query heads that share one KV head
-// form M = N*G query rows; a CTA owns a tile of those rows and one slice of the
-// context (split-K), streams the slice's pages once, keeps an online softmax in
-// fp32 and accumulates P.V in fp32.  Partial (m, l, O) of the slices are merged by
-// a second kernel.  Key tile = one 64-token page.
+// Flash-decoding layout.  The N tree nodes x G query heads that share one KV head
+// form M = N*G query rows (<= 512).  A CTA owns up to two 128-row tiles of them and
+// one slice of the context (split-K).  Per 128-key tile (two 64-token pages):
+//   TMA      : K and V pages -> 128B-swizzled shared memory, 5-slot ring, mbarriers
+//   tcgen05  : S_t = Q_t K^T into TMEM (fp32), one elected thread issues
+//   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S, online
+//              softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back into TMEM
+//   tcgen05  : O_t += P_t V with P as the TMEM A operand, V MN-major from shared memory
+// TMEM map (512 columns): S0/P0 [0,128) S1/P1 [128,256) O0 [256,384) O1 [384,512).
+// Slices are merged by attention_merge_kernel (warp per output row).  All waits are
+// bounded: on expiry the CTA records SAGE_STATUS_TIMEOUT, drains its copies, frees its
+// TMEM and returns.
+#include <cuda.h>
+
 #include "sage_common.cuh"
 
 namespace sage {
 
-constexpr int kRowsPerCta = 128;
-constexpr int kAttnThreads = 256;            // 8 warps x 16 rows
-constexpr int kTileBytes = kPageSize * kHeadDim * 2;   // 16 KB per K or V page tile
-constexpr int kStages = 2;
+constexpr int kTileKeys = 128;                 // keys per pipeline step (two pages)
+constexpr int kRowTile = 128;                  // query rows per MMA tile
+constexpr int kRowsPerCta = 2 * kRowTile;
+constexpr int kSlots = 5;                      // K/V ring: K0 V0 K1 V1 K2 ...
+constexpr int kSlotBytes = kTileKeys * kHeadDim * 2;        // 32 KB
+constexpr int kHalfBytes = kTileKeys * 64 * 2;              // one 64-wide d-half of a tile: 16 KB
+constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // 8 KB
+constexpr int kQTileBytes = kRowTile * kHeadDim * 2;        // 32 KB
+constexpr int kAttnThreads = 320;              // 2 softmax warpgroups + TMA warp + MMA warp
+constexpr int kSmemBytes = 2 * kQTileBytes + kSlots * kSlotBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: far beyond any legitimate wait
 
 struct AttnParams {
     const __nv_bfloat16* q;
-    const __nv_bfloat16* k_pool;
-    const __nv_bfloat16* v_pool;
     __nv_bfloat16* out;
     float* part_o;     // [layer][split][sum_nodes*Hq][128]   unnormalised
-    float* part_ml;    // [layer][split][sum_nodes*Hq][2]     (m in log2 units, l)
+    float* part_ml;    // [layer][split][sum_nodes*Hq][2]     (reference max in log2 units, l)
     const int32_t* page_table;
     const int32_t* seq_len;
     const int32_t* parent;
     const int32_t* node_offsets;
     int32_t* status;
-    int64_t layer_stride;
     int n_layers, batch, sum_nodes, n_pages, max_pages;
     int Hq, Hkv, G, n_splits;
     float scale_log2;  // sm_scale * log2(e)
 };
 
+struct __align__(8) Barriers {
+    uint64_t full[kSlots];
+    uint64_t empty[kSlots];
+    uint64_t s_full[2];
+    uint64_t p_full[2];
+    uint64_t o_full;
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
-    const int sz = valid ? 16 : 0;   // size 0: the 16 destination bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz));
+// ---- mbarrier ---------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* bars, int32_t* status) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (bars->abort) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            bars->abort = 1;
+            report_status(status, SAGE_STATUS_TIMEOUT);
+            return false;
+        }
+    }
+}
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+// ---- TMA ----------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+
+// ---- tcgen05 --------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (quadrant*32 + i)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Tile byte offset of (key row, 16-byte chunk) with an XOR swizzle against bank conflicts.
-__device__ __forceinline__ uint32_t tile_off(int key, int chunk) { return key * 256 + ((chunk ^ (key & 7)) << 4); }
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
+// offsets in 16-byte units, version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = 128.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;                    // A, B both K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);       // B (= V) MN-major
 
-__global__ void __launch_bounds__(kAttnThreads, 1) tree_attention_kernel(AttnParams p) {
-    extern __shared__ __align__(128) uint8_t smem[];
+__global__ void __launch_bounds__(kAttnThreads, 1)
+tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
+    extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_anc[SAGE_MAX_NODES];
     __shared__ int s_flag;
-    uint8_t* sK = smem;                          // [kStages][16 KB]
-    uint8_t* sV = smem + kStages * kTileBytes;   // [kStages][16 KB]
+    // 1024-byte alignment: the 128B swizzle pattern repeats every 1024 bytes of address
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;                                 // [2 tiles][2 d-halves][128 rows][128 B]
+    uint8_t* sKV = smem + 2 * kQTileBytes;              // [kSlots][2 d-halves][128 keys][128 B]
+    Barriers* bars = reinterpret_cast<Barriers*>(sKV + kSlots * kSlotBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int split = blockIdx.x, rtile = blockIdx.y;
+    const int split = blockIdx.x, rpair = blockIdx.y;
     const int g = blockIdx.z % p.Hkv;
     const int b = (blockIdx.z / p.Hkv) % p.batch;
     const int layer = blockIdx.z / (p.Hkv * p.batch);
 
+    // ---- uniform early exits (before any barrier or TMEM is touched)
     const int n0 = p.node_offsets[b];
     const int N = p.node_offsets[b + 1] - n0;
     const int L = p.seq_len[b];
-    if (tid == 0) s_flag = 0;
-    __syncthreads();
     if (N < 1 || N > SAGE_MAX_NODES || n0 < 0 || n0 + N > p.sum_nodes) {
         if (tid == 0) report_status(p.status, SAGE_STATUS_BAD_TREE);
         return;
@@ -92,9 +197,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) tree_attention_kernel(AttnPar
         return;
     }
     const int M = N * p.G;
-    if (rtile * kRowsPerCta >= M) return;
+    if (rpair * kRowsPerCta >= M) return;
+    const int n_rtiles = (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1;
 
-    // ancestor bitsets of this tree
+    if (tid == 0) s_flag = 0;
+    __syncthreads();
     if (tid < SAGE_MAX_NODES) {
         uint64_t a = 0;
         if (tid < N) {
@@ -104,199 +211,295 @@ __global__ void __launch_bounds__(kAttnThreads, 1) tree_attention_kernel(AttnPar
         }
         s_anc[tid] = a;
     }
-    __syncthreads();
-    if (s_flag) {
-        if (tid == 0) report_status(p.status, SAGE_STATUS_BAD_TREE);
-        return;
-    }
-
-    const int n_tiles = (T + kPageSize - 1) / kPageSize;
+    const int n_pages_seq = (T + kPageSize - 1) / kPageSize;
+    const int n_tiles = (T + kTileKeys - 1) / kTileKeys;
     const int per_split = (n_tiles + p.n_splits - 1) / p.n_splits;
     const int t_begin = split * per_split;
     const int t_end = min(n_tiles, t_begin + per_split);
-
-    // the two rows this thread owns inside its warp's 16-row slab
-    const int r_lo = rtile * kRowsPerCta + warp * 16 + (lane >> 2);
-    const int r_hi = r_lo + 8;
-    const bool v_lo = r_lo < M, v_hi = r_hi < M;
-    const int node_lo = v_lo ? r_lo / p.G : 0, node_hi = v_hi ? r_hi / p.G : 0;
-    const int h_lo = g * p.G + (v_lo ? r_lo % p.G : 0), h_hi = g * p.G + (v_hi ? r_hi % p.G : 0);
-    const size_t qrow_lo = ((size_t)layer * p.sum_nodes + n0 + node_lo) * p.Hq + h_lo;
-    const size_t qrow_hi = ((size_t)layer * p.sum_nodes + n0 + node_hi) * p.Hq + h_hi;
-    const uint64_t anc_lo = s_anc[node_lo], anc_hi = s_anc[node_hi];
-
-    // Q fragments (A operand, 16 rows x 128 d): 8 k-steps x 4 registers
-    uint32_t qf[8][4];
-    {
-        const uint32_t* qlo = reinterpret_cast<const uint32_t*>(p.q + qrow_lo * kHeadDim);
-        const uint32_t* qhi = reinterpret_cast<const uint32_t*>(p.q + qrow_hi * kHeadDim);
-        const int c = lane & 3;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            qf[ks][0] = v_lo ? qlo[ks * 8 + c] : 0u;
-            qf[ks][1] = v_hi ? qhi[ks * 8 + c] : 0u;
-            qf[ks][2] = v_lo ? qlo[ks * 8 + 4 + c] : 0u;
-            qf[ks][3] = v_hi ? qhi[ks * 8 + 4 + c] : 0u;
-        }
+    const int nt = max(0, t_end - t_begin);
+    // page ids of this slice must be valid before the TMA warp uses them as coordinates
+    for (int pg = t_begin * 2 + tid; pg < min(t_end * 2, n_pages_seq); pg += kAttnThreads) {
+        const int id = p.page_table[(size_t)b * p.max_pages + pg];
+        if (id < 0 || id >= p.n_pages) s_flag = 2;
+    }
+    __syncthreads();
+    if (s_flag) {
+        if (tid == 0) report_status(p.status, s_flag == 1 ? SAGE_STATUS_BAD_TREE : SAGE_STATUS_BAD_PAGE);
+        return;
     }
 
-    float o[16][4];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-
-    const __nv_bfloat16* kbase = p.k_pool + (int64_t)layer * p.layer_stride;
-    const __nv_bfloat16* vbase = p.v_pool + (int64_t)layer * p.layer_stride;
-
-    auto load_tile = [&](int t, int stage) {
-        int page = p.page_table[(size_t)b * p.max_pages + t];
-        if (page < 0 || page >= p.n_pages) {
-            report_status(p.status, SAGE_STATUS_BAD_PAGE);
-            page = 0;
-        }
-        const int64_t off = ((int64_t)page * p.Hkv + g) * (kPageSize * kHeadDim);
-        const int valid_keys = min(kPageSize, T - t * kPageSize);
-        const uint32_t dk = smem_u32(sK + stage * kTileBytes), dv = smem_u32(sV + stage * kTileBytes);
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int c = tid + it * kAttnThreads;      // 1024 chunks of 16 bytes
-            const int key = c >> 4, ch = c & 15;
-            const bool ok = key < valid_keys;
-            cp_async_16(dk + tile_off(key, ch), kbase + off + key * kHeadDim + ch * 8, ok);
-            cp_async_16(dv + tile_off(key, ch), vbase + off + key * kHeadDim + ch * 8, ok);
-        }
-    };
-
-    if (t_begin < t_end) load_tile(t_begin, 0);
-    cp_async_commit();
-
-    for (int t = t_begin; t < t_end; ++t) {
-        const int stage = (t - t_begin) & 1;
-        if (t + 1 < t_end) load_tile(t + 1, stage ^ 1);
-        cp_async_commit();
-        cp_async_wait<1>();
-        __syncthreads();
-
-        const uint32_t kaddr = smem_u32(sK + stage * kTileBytes), vaddr = smem_u32(sV + stage * kTileBytes);
-        // S = Q K^T : 16 rows x 64 keys
-        float s[8][4];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-            for (int np = 0; np < 4; ++np) {
-                const int key = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                const int ch = ks * 2 + ((lane >> 3) & 1);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4(kaddr + tile_off(key, ch), b0, b1, b2, b3);
-                mma_bf16_16816(s[np * 2], qf[ks], b0, b1);
-                mma_bf16_16816(s[np * 2 + 1], qf[ks], b2, b3);
+    // ---- set-up: barriers, TMEM, Q tiles
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+        for (int t = 0; t < 2; ++t) { mbar_init(&bars->s_full[t], 1); mbar_init(&bars->p_full[t], kRowTile); }
+        mbar_init(&bars->o_full, 1);
+        bars->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp < 8) {
+        // Q rows -> K-major 128B-swizzled tiles; rows past M are zero
+        for (int c = tid; c < n_rtiles * kRowTile * 16; c += 256) {
+            const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
+            const int R = rpair * kRowsPerCta + t * kRowTile + r;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (R < M) {
+                const size_t row = ((size_t)layer * p.sum_nodes + n0 + R / p.G) * p.Hq + g * p.G + R % p.G;
+                v = *reinterpret_cast<const uint4*>(p.q + row * kHeadDim + ch * 8);
             }
+            const int half = ch >> 3, cc = ch & 7;
+            *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
         }
-        // scale to log2 units and mask the tree part of the tile
-        const int pos0 = t * kPageSize;
-        const bool need_mask = pos0 + kPageSize > L;
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float v = s[nt][e] * p.scale_log2;
-                if (need_mask) {
-                    const int j = pos0 + nt * 8 + (lane & 3) * 2 + (e & 1) - L;   // tree slot, <0 = prefix
-                    const uint64_t anc = (e < 2) ? anc_lo : anc_hi;
-                    const bool vis = j < 0 || (j < N && ((anc >> j) & 1ull));
-                    v = vis ? v : -INFINITY;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA unit
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    if (warp == 8) {
+        // =========================== TMA producer ===========================
+        if (lane == 0) {
+            int issued = 0;
+            for (int n = 0; n < 2 * nt; ++n) {
+                const int slot = n % kSlots, use = n / kSlots;
+                if (use > 0 && !mbar_wait(&bars->empty[slot], (use - 1) & 1, bars, p.status)) break;
+                const int tile = t_begin + (n >> 1);
+                const CUtensorMap* map = (n & 1) ? &vmap : &kmap;
+                const int pg0 = tile * 2;
+                const int n_pg = min(2, n_pages_seq - pg0);
+                mbar_expect_tx(&bars->full[slot], (uint32_t)n_pg * 2 * kPageHalfBytes);
+                const uint32_t dst = smem_u32(sKV + slot * kSlotBytes);
+                for (int pp = 0; pp < n_pg; ++pp) {
+                    const int id = p.page_table[(size_t)b * p.max_pages + pg0 + pp];
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_4d(dst + h * kHalfBytes + pp * kPageHalfBytes, map, h * 64, 0, id * p.Hkv + g, layer,
+                                    &bars->full[slot]);
                 }
-                s[nt][e] = v;
+                issued = n + 1;
+            }
+            if (bars->abort) {
+                // drain: every issued copy must land before the CTA may exit
+                for (int n = max(0, issued - kSlots); n < issued; ++n) {
+                    const long long t0 = clock64();
+                    while (!mbar_try(&bars->full[n % kSlots], (n / kSlots) & 1) && clock64() - t0 < kWaitCycles) {}
+                }
             }
         }
-        float mx_lo = -INFINITY, mx_hi = -INFINITY;
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
-            mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
+    } else if (warp == 9) {
+        // =========================== MMA issuer ===========================
+        const uint32_t q_addr = smem_u32(sQ), kv_addr = smem_u32(sKV);
+        auto issue_qk = [&](int t, int slot) {
+            // S_t = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                mma_ss(tmem + t * 128, make_desc(q_addr + t * kQTileBytes + off, 16, 1024),
+                       make_desc(kv_addr + slot * kSlotBytes + off, 16, 1024), kIdescQK, ks > 0);
+            }
+        };
+        auto issue_pv = [&](int t, int slot, bool first) {
+            // O_t += P_t V: 8 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + ks * 8,
+                       make_desc(kv_addr + slot * kSlotBytes + ks * 2048, kHalfBytes, 1024), kIdescPV,
+                       (!first || ks > 0));
+        };
+        // lane 0 polls, the result is broadcast so that the warp never diverges on a wait
+        auto wait_all = [&](uint64_t* bar, uint32_t parity) {
+            int r = 1;
+            if (lane == 0) r = mbar_wait(bar, parity, bars, p.status) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, r, 0) != 0;
+        };
+        bool ok = nt > 0;
+        if (ok) ok = wait_all(&bars->full[0], 0);
+        if (ok) {
+            tc_fence_after();
+            if (lane == 0) {
+                for (int t = 0; t < n_rtiles; ++t) { issue_qk(t, 0); tc_commit(&bars->s_full[t]); }
+                tc_commit(&bars->empty[0]);
+            }
+            __syncwarp();
         }
-        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-        const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-        const float base_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, base_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
-        const float a_lo = exp2f(m_lo - base_lo), a_hi = exp2f(m_hi - base_hi);
-        m_lo = mn_lo; m_hi = mn_hi;
-        float sum_lo = 0.f, sum_hi = 0.f;
-        uint32_t pf[4][4];                         // P as A fragments: 4 k-steps of 16 keys
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            const float p0 = exp2f(s[nt][0] - base_lo), p1 = exp2f(s[nt][1] - base_lo);
-            const float p2 = exp2f(s[nt][2] - base_hi), p3 = exp2f(s[nt][3] - base_hi);
-            sum_lo += p0 + p1;
-            sum_hi += p2 + p3;
-            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
-        }
-        sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1);
-        sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
-        sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1);
-        sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
-        l_lo = l_lo * a_lo + sum_lo;
-        l_hi = l_hi * a_hi + sum_hi;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { o[i][0] *= a_lo; o[i][1] *= a_lo; o[i][2] *= a_hi; o[i][3] *= a_hi; }
-        // O += P V : k over 64 keys (4 steps), n over 128 d (16 tiles)
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-#pragma unroll
-            for (int np = 0; np < 8; ++np) {
-                const int key = ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                const int ch = np * 2 + (lane >> 4);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(vaddr + tile_off(key, ch), b0, b1, b2, b3);
-                mma_bf16_16816(o[np * 2], pf[ks], b0, b1);
-                mma_bf16_16816(o[np * 2 + 1], pf[ks], b2, b3);
+        for (int j = 0; ok && j < nt; ++j) {
+            const int nv = 2 * j + 1, vslot = nv % kSlots;
+            ok = wait_all(&bars->full[vslot], (nv / kSlots) & 1);
+            if (!ok) break;
+            const int valid = min(kTileKeys, T - (t_begin + j) * kTileKeys);
+            if (valid < kTileKeys) {
+                // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
+                uint8_t* vb = sKV + vslot * kSlotBytes;
+                for (int c = lane; c < (kTileKeys - valid) * 16; c += 32) {
+                    const int r = valid + c / 16, ch = c % 16;
+                    *reinterpret_cast<uint4*>(vb + (ch >> 3) * kHalfBytes + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
+            const int nk = 2 * (j + 1), kslot = nk % kSlots;
+            for (int t = 0; ok && t < n_rtiles; ++t) {
+                ok = wait_all(&bars->p_full[t], j & 1);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    issue_pv(t, vslot, j == 0);
+                    if (t == n_rtiles - 1) tc_commit(&bars->empty[vslot]);
+                }
+                if (j + 1 < nt) {
+                    if (t == 0) {
+                        ok = wait_all(&bars->full[kslot], (nk / kSlots) & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+                    if (lane == 0) {
+                        issue_qk(t, kslot);
+                        tc_commit(&bars->s_full[t]);
+                        if (t == n_rtiles - 1) tc_commit(&bars->empty[kslot]);
+                    }
+                }
+                __syncwarp();
             }
         }
-        __syncthreads();   // everyone is done with this stage before it is refilled
-    }
-    cp_async_wait<0>();
-
-    // ---- epilogue
-    const int c2 = (lane & 3) * 2;
-    if (p.n_splits == 1) {
-        const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
-        if (v_lo) {
-            uint32_t* dst = reinterpret_cast<uint32_t*>(p.out + qrow_lo * kHeadDim);
-#pragma unroll
-            for (int nt = 0; nt < 16; ++nt) dst[(nt * 8 + c2) >> 1] = pack_bf16(o[nt][0] * inv_lo, o[nt][1] * inv_lo);
-        }
-        if (v_hi) {
-            uint32_t* dst = reinterpret_cast<uint32_t*>(p.out + qrow_hi * kHeadDim);
-#pragma unroll
-            for (int nt = 0; nt < 16; ++nt) dst[(nt * 8 + c2) >> 1] = pack_bf16(o[nt][2] * inv_hi, o[nt][3] * inv_hi);
-        }
+        if (lane == 0) tc_commit(&bars->o_full);      // arrives when every MMA above has completed
+        __syncwarp();
     } else {
-        const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
-        const size_t slab = ((size_t)layer * p.n_splits + split) * rows_total;
-        if (v_lo) {
-            const size_t r = slab + (size_t)(n0 + node_lo) * p.Hq + h_lo;
-            float2* dst = reinterpret_cast<float2*>(p.part_o + r * kHeadDim);
+        // =========================== softmax warpgroups ===========================
+        const int t = warp >> 2;                        // row tile of this warpgroup
+        const int r = tid & 127;                        // row inside the tile == TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_taddr = tmem + lane_base + t * 128;
+        const uint32_t o_taddr = tmem + lane_base + 256 + t * 128;
+        const int R = rpair * kRowsPerCta + t * kRowTile + r;
+        const bool row_ok = R < M;
+        const int node = row_ok ? R / p.G : 0;
+        const uint64_t anc = s_anc[node];
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = (t < n_rtiles);
+        for (int j = 0; ok && j < nt; ++j) {
+            ok = mbar_wait(&bars->s_full[t], j & 1, bars, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[4][32];
 #pragma unroll
-            for (int nt = 0; nt < 16; ++nt) dst[(nt * 8 + c2) >> 1] = make_float2(o[nt][0], o[nt][1]);
-            if ((lane & 3) == 0) { p.part_ml[r * 2] = m_lo; p.part_ml[r * 2 + 1] = l_lo; }
-        }
-        if (v_hi) {
-            const size_t r = slab + (size_t)(n0 + node_hi) * p.Hq + h_hi;
-            float2* dst = reinterpret_cast<float2*>(p.part_o + r * kHeadDim);
+            for (int c = 0; c < 4; ++c) tmem_ld32(s_taddr + c * 32, sr[c]);
+            tmem_wait_ld();
+            const int pos0 = (t_begin + j) * kTileKeys;
+            if (pos0 + kTileKeys > L) {
+                // tile reaches into the tree part (or past the end): apply the ancestor mask
 #pragma unroll
-            for (int nt = 0; nt < 16; ++nt) dst[(nt * 8 + c2) >> 1] = make_float2(o[nt][2], o[nt][3]);
-            if ((lane & 3) == 0) { p.part_ml[r * 2] = m_hi; p.part_ml[r * 2 + 1] = l_hi; }
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int jt = pos0 + c * 32 + i - L;        // tree slot; < 0 = prefix
+                        const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
+                        if (!vis) sr[c][i] = 0xff800000u;             // -inf
+                    }
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[c][i]));
+            const float m_cand = mx * p.scale_log2;
+            // lazy rescale: move the reference only when the row max grew by more than 2^8
+            const bool grow = m_cand > m_ref + 8.0f;
+            float alpha = 1.0f;
+            if (grow) {
+                alpha = fast_exp2(m_ref - m_cand);          // 0 when m_ref was -inf
+                m_ref = m_cand;
+            }
+            const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                // O_t *= alpha.  The commit that signalled s_full covers every earlier MMA, so PV(j-1) is done.
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t orr[32];
+                    tmem_ld32(o_taddr + c * 32, orr);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+                    tmem_st32(o_taddr + c * 32, orr);
+                }
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * i]), p.scale_log2, neg_ref));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * i + 1]), p.scale_log2, neg_ref));
+                    sum += p0 + p1;
+                    pk[i] = pack_bf16(p0, p1);
+                }
+                tmem_st16(s_taddr + c * 16, pk);            // P_t (bf16 pairs) over the first 64 columns of S_t
+            }
+            l_sum = l_sum * alpha + sum;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars->p_full[t]);
         }
+        // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
+        if (t < n_rtiles) {
+            if (nt > 0 && ok) ok = mbar_wait(&bars->o_full, 0, bars, p.status);
+            if (ok) tc_fence_after();
+            const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
+            const size_t row = (size_t)(n0 + node) * p.Hq + g * p.G + (row_ok ? R % p.G : 0);
+            const float inv = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
+            float* po = nullptr;
+            __nv_bfloat16* oo = nullptr;
+            if (p.n_splits == 1) {
+                oo = p.out + ((size_t)layer * rows_total + row) * kHeadDim;
+            } else {
+                const size_t pr = ((size_t)layer * p.n_splits + split) * rows_total + row;
+                po = p.part_o + pr * kHeadDim;
+                if (row_ok && ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = (nt > 0) ? l_sum : 0.f; }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t orr[32];
+                if (nt > 0 && ok) {
+                    tmem_ld32(o_taddr + c * 32, orr);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) orr[i] = 0u;
+                }
+                if (row_ok && ok) {
+                    if (oo) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 v;
+                            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+                            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+                            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+                            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+                            *reinterpret_cast<uint4*>(oo + c * 32 + i * 8) = v;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            *reinterpret_cast<uint4*>(po + c * 32 + i * 4) =
+                                make_uint4(orr[4 * i], orr[4 * i + 1], orr[4 * i + 2], orr[4 * i + 3]);
+                    }
+                }
+            }
+        }
+    }
+    // ---- teardown: every role is past its last TMEM access
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     }
 }
 
 // Split-K merge: one warp per (layer, node, head) row.  Lanes first reduce (m, l) over
-// the splits with shuffles, then each lane combines its four output columns.
+// the slices with shuffles, then each lane combines its four output columns.
 __global__ void attention_merge_kernel(AttnParams p) {
     const int warps = blockDim.x >> 5;
     const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
@@ -312,9 +515,9 @@ __global__ void attention_merge_kernel(AttnParams p) {
         m = p.part_ml[r * 2];
         l = p.part_ml[r * 2 + 1];
     }
-    float mx = m;
+    float mx = (l > 0.f) ? m : -INFINITY;
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    const float w = (l > 0.f) ? exp2f(m - mx) : 0.f;   // weight of this lane's split
+    const float w = (l > 0.f) ? exp2f(m - mx) : 0.f;   // weight of this lane's slice
     float lsum = l * w;
     for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -334,15 +537,56 @@ __global__ void attention_merge_kernel(AttnParams p) {
 }
 
 static int pick_splits(int n_layers, int batch, int n_kv_heads, int G, int max_pages) {
-    // enough CTAs for ~2 waves of 148 SMs, at least 4 pages per slice, at most 32 slices
-    const int row_tiles = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
-    const long base = (long)n_layers * batch * n_kv_heads * row_tiles;
-    long s = (2 * 148 + base - 1) / base;
-    const int by_len = max_pages / 4 > 0 ? max_pages / 4 : 1;
-    if (s > by_len) s = by_len;
-    if (s > 32) s = 32;
-    if (s < 1) s = 1;
-    return (int)s;
+    // One CTA is resident per SM.  Take the smallest slice count whose CTA count fills whole
+    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 4 key tiles per slice.
+    const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
+    const long base = (long)n_layers * batch * n_kv_heads * row_pairs;
+    const int tiles = (max_pages + 1) / 2;
+    int s_max = tiles / 4;
+    if (s_max > 32) s_max = 32;
+    if (s_max < 1) s_max = 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= s_max; ++s) {
+        const long ctas = base * s;
+        const double eff = (double)ctas / (148.0 * ((ctas + 147) / 148));
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
+        if (eff >= 0.9) { best = s; break; }
+    }
+    return best;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// Pool viewed as [layer][page*Hkv + head][slot][d]; one box = one 64-wide d-half of one (page, head).
+static bool make_pool_map(CUtensorMap* map, const void* pool, int n_layers, int n_pages, int n_kv_heads,
+                          int64_t layer_stride_elems) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t page_head_bytes = (cuuint64_t)kPageSize * kHeadDim * 2;
+    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)kPageSize, (cuuint64_t)n_pages * n_kv_heads,
+                          (cuuint64_t)n_layers};
+    cuuint64_t layer_bytes = n_layers > 1 ? (cuuint64_t)layer_stride_elems * 2 : dims[2] * page_head_bytes;
+    cuuint64_t strides[3] = {(cuuint64_t)kHeadDim * 2, page_head_bytes, layer_bytes};
+    cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace sage
@@ -375,32 +619,38 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     if ((long)n_layers * batch * n_kv_heads > 65535) return SAGE_ERR_UNSUPPORTED;
     if ((((uintptr_t)q | (uintptr_t)k_pool | (uintptr_t)v_pool | (uintptr_t)out) & 15) || (layer_stride_elems & 7))
         return SAGE_ERR_INVALID_ARG;
+    if (n_layers > 1 && layer_stride_elems < (int64_t)n_pages * n_kv_heads * kPageSize * kHeadDim)
+        return SAGE_ERR_INVALID_ARG;
     if (batch == 0) return SAGE_OK;
     const int S = pick_splits(n_layers, batch, n_kv_heads, G, max_pages_per_seq);
     const size_t need = sage_tree_attention_workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads,
                                                            head_dim, max_pages_per_seq);
     if (S > 1 && (!ws || ws_bytes < need || ((uintptr_t)ws & 15))) return SAGE_ERR_WORKSPACE;
     AttnParams p{};
-    p.q = (const __nv_bfloat16*)q; p.k_pool = (const __nv_bfloat16*)k_pool; p.v_pool = (const __nv_bfloat16*)v_pool;
+    p.q = (const __nv_bfloat16*)q;
     p.out = (__nv_bfloat16*)out;
     p.part_o = (float*)ws;
     p.part_ml = S > 1 ? (float*)ws + (size_t)n_layers * S * sum_nodes * n_q_heads * kHeadDim : nullptr;
     p.page_table = page_table; p.seq_len = seq_len; p.parent = parent; p.node_offsets = node_offsets;
-    p.status = status; p.layer_stride = layer_stride_elems;
+    p.status = status;
     p.n_layers = n_layers; p.batch = batch; p.sum_nodes = sum_nodes; p.n_pages = n_pages;
     p.max_pages = max_pages_per_seq; p.Hq = n_q_heads; p.Hkv = n_kv_heads; p.G = G; p.n_splits = S;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
 
+    CUtensorMap kmap, vmap;
+    if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
+        !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
+        return SAGE_ERR_CUDA;
     static bool attr_set = false;
-    const int smem = 2 * kStages * kTileBytes;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tree_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(tree_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
             return SAGE_ERR_CUDA;
         attr_set = true;
     }
-    const int row_tiles = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
-    dim3 grid(S, row_tiles, n_layers * batch * n_kv_heads);
-    tree_attention_kernel<<<grid, kAttnThreads, smem, as_stream(stream)>>>(p);
+    const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
+    dim3 grid(S, row_pairs, n_layers * batch * n_kv_heads);
+    tree_attention_kernel<<<grid, kAttnThreads, kSmemBytes, as_stream(stream)>>>(p, kmap, vmap);
     if (S > 1) {
         const size_t rows_total = (size_t)sum_nodes * n_q_heads;
         dim3 mg((unsigned)((rows_total + 7) / 8), n_layers);
