@@ -48,6 +48,7 @@ extern "C" {
 #define SAGE_ERR_UNSUPPORTED  2   /* outside the supported envelope                     */
 #define SAGE_ERR_WORKSPACE    3   /* ws == NULL or ws_bytes too small                   */
 #define SAGE_ERR_CUDA         4   /* a CUDA runtime / driver call failed                */
+#define SAGE_ERR_TOO_LARGE    5   /* problem needs more scratch than the built-in array */
 
 /* values written to the device status word (first error wins) */
 #define SAGE_STATUS_BAD_TREE  101 /* parent array / node count violates the tree rules  */
@@ -95,6 +96,35 @@ int sage_expand_topk(const float *logits, int rows, int vocab, int64_t row_strid
                      int batch, const int32_t *root_token, int32_t *draft_token,
                      void *ws, size_t ws_bytes, int32_t *status, void *stream);
 size_t sage_expand_topk_workspace_size(int rows, int vocab);
+
+/* sage_expand_topk for callers that cannot provide scratch memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, not another operation.)
+ * Who needs it: code that runs where no device allocation is possible -- a plug-in that is
+ * handed only its input and output buffers by a serving engine whose own pool already owns
+ * all of the GPU's memory, or a decode loop that must not call cudaMalloc because that call
+ * synchronises the whole device.  Such a caller has nowhere to get `ws` from.
+ * Same arguments, results and error codes as sage_expand_topk, minus ws / ws_bytes: the
+ * scratch is a fixed array of SAGE_STATIC_SCRATCH_BYTES bytes inside the library, present on
+ * every GPU that loads the library, for the life of the process.  The call performs no
+ * allocation of any kind.
+ *  - Limit: sage_expand_topk_workspace_size(rows, vocab) must not exceed
+ *    SAGE_STATIC_SCRATCH_BYTES (60 rows x 152064 need about 90 KB; several thousand rows
+ *    fit); otherwise SAGE_ERR_TOO_LARGE is returned and nothing is enqueued.
+ *  - The first call on each device looks up the array's device address (a runtime query,
+ *    done with that device current, which also loads the library's kernels there).  Make
+ *    that first call before starting any stream capture on that device.
+ *  - All calls on one device use the same array, and it keeps whatever the previous call
+ *    left; the kernels overwrite every slot they later read, so no clearing is needed.  Two
+ *    calls that may run at the same time on one GPU (different streams, or different host
+ *    threads) race on the array and give wrong results: keep them ordered on one stream. */
+#define SAGE_STATIC_SCRATCH_BYTES (1 << 20)
+int sage_expand_topk_static(const float *logits, int rows, int vocab, int64_t row_stride,
+                            int k, int k_entropy,
+                            int32_t *topk_idx, float *topk_logprob,
+                            float *entropy_full, float *entropy_topk, float *alpha, float *lse,
+                            const int32_t *parent, const int32_t *rank, const int32_t *node_offsets,
+                            int batch, const int32_t *root_token, int32_t *draft_token,
+                            int32_t *status, void *stream);
 
 /* Confidence -> tree template (Eq. 10, Eq. 11; Algorithm 1 "Phase 3: Dynamic Tree
  * Update").  For sequence b the confidence is alpha[alpha_row ? alpha_row[b] : b]

@@ -22,6 +22,8 @@ SAGE_ERR_INVALID_ARG = 1
 SAGE_ERR_UNSUPPORTED = 2
 SAGE_ERR_WORKSPACE = 3
 SAGE_ERR_CUDA = 4
+SAGE_ERR_TOO_LARGE = 5
+SAGE_STATIC_SCRATCH_BYTES = 1 << 20
 SAGE_STATUS_BAD_TREE = 101
 SAGE_STATUS_BAD_PAGE = 102
 SAGE_STATUS_TIMEOUT = 103
@@ -57,6 +59,9 @@ _lib.sage_expand_topk.argtypes = [_vp, _i, _i, _i64, _i, _i, _vp, _vp, _vp, _vp,
                                   _vp, _vp, _vp, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.sage_expand_topk_workspace_size.restype = _sz
 _lib.sage_expand_topk_workspace_size.argtypes = [_i, _i]
+_lib.sage_expand_topk_static.restype = _i
+_lib.sage_expand_topk_static.argtypes = [_vp, _i, _i, _i64, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp,
+                                         _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp]
 _lib.sage_select_tree.restype = _i
 _lib.sage_select_tree.argtypes = [_vp, _vp, _i, ctypes.POINTER(SagePolicy), _vp, _vp, _vp,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -147,6 +152,28 @@ def sage_expand_topk(logits: torch.Tensor, k: int, k_entropy: int, *, parent=Non
                                  _ptr(o.get("draft_token")), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
     _check(code, "sage_expand_topk")
     return o
+
+
+def sage_expand_topk_static(logits: torch.Tensor, k: int, k_entropy: int, *, parent=None, rank=None,
+                            node_offsets=None, root_token=None, out: Dict[str, torch.Tensor],
+                            status: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """sage_expand_topk without a workspace argument, for callers that cannot allocate device
+    memory: the scratch is an array inside the library.  To honour that, this wrapper
+    allocates nothing either -- every output tensor must already be in ``out`` (topk_idx,
+    topk_logprob, entropy_full, entropy_topk, alpha, lse, and draft_token when the tree
+    arrays are given).  Calls on one GPU must not overlap; problems whose workspace would
+    exceed SAGE_STATIC_SCRATCH_BYTES raise SageError(SAGE_ERR_TOO_LARGE)."""
+    assert logits.dtype == torch.float32 and logits.dim() == 2 and logits.stride(1) == 1
+    rows, vocab = logits.shape
+    batch = node_offsets.numel() - 1 if parent is not None else 0
+    code = _lib.sage_expand_topk_static(logits.data_ptr(), rows, vocab, logits.stride(0), k, k_entropy,
+                                        _ptr(out["topk_idx"]), _ptr(out["topk_logprob"]),
+                                        _ptr(out["entropy_full"]), _ptr(out["entropy_topk"]), _ptr(out["alpha"]),
+                                        _ptr(out["lse"]), _ptr(parent), _ptr(rank), _ptr(node_offsets), batch,
+                                        _ptr(root_token), _ptr(out.get("draft_token")), _ptr(status),
+                                        _stream(stream))
+    _check(code, "sage_expand_topk_static")
+    return out
 
 
 def sage_select_tree(alpha: torch.Tensor, policy: SagePolicy, *, alpha_row=None, batch: Optional[int] = None,

@@ -14,6 +14,8 @@
 // lists, then derives lse, full entropy, log-probs, top-k entropy and alpha.
 #include <math.h>
 
+#include <mutex>
+
 #include "sage_common.cuh"
 
 namespace sage {
@@ -336,4 +338,59 @@ extern "C" int sage_expand_topk(const float* logits, int rows, int vocab, int64_
         expand_gather_kernel<<<batch, 64, 0, as_stream(stream)>>>(topk_idx, k, rows, parent, rank, node_offsets,
                                                                   root_token, draft_token, status);
     return launch_status();
+}
+
+// ---------------------------------------------------------------------------
+// sage_expand_topk_static: the same computation with the scratch memory built
+// into the library instead of supplied by the caller.
+// ---------------------------------------------------------------------------
+namespace sage {
+
+// Scratch of the static variant.  It is part of the library image: every GPU on which
+// the library's kernels get loaded holds these bytes until the process exits.
+__device__ __align__(256) static unsigned char g_static_scratch[SAGE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+
+// Device address of g_static_scratch on the current device (nullptr on failure).  In host
+// code the array's name is only a handle for the runtime, not a device address, so the
+// address is looked up once per device, with that device current, and remembered.
+static void* static_scratch_address() {
+    static std::mutex mu;
+    static void* addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        addr[dev] = p;
+    }
+    return addr[dev];
+}
+
+}  // namespace sage
+
+extern "C" int sage_expand_topk_static(const float* logits, int rows, int vocab, int64_t row_stride, int k,
+                                       int k_entropy, int32_t* topk_idx, float* topk_logprob, float* entropy_full,
+                                       float* entropy_topk, float* alpha, float* lse, const int32_t* parent,
+                                       const int32_t* rank, const int32_t* node_offsets, int batch,
+                                       const int32_t* root_token, int32_t* draft_token, int32_t* status,
+                                       void* stream) {
+    if (rows < 0 || vocab < 1) return SAGE_ERR_INVALID_ARG;
+    if (rows > 0 && sage_expand_topk_workspace_size(rows, vocab) > (size_t)SAGE_STATIC_SCRATCH_BYTES)
+        return SAGE_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    if (rows > 0) {
+        scratch = static_scratch_address();
+        if (scratch == nullptr) return SAGE_ERR_CUDA;
+    }
+    // Every scratch slot the finalize kernel reads is written by the partial kernel of the
+    // same call, so nothing has to be cleared between calls.
+    return sage_expand_topk(logits, rows, vocab, row_stride, k, k_entropy, topk_idx, topk_logprob, entropy_full,
+                            entropy_topk, alpha, lse, parent, rank, node_offsets, batch, root_token, draft_token,
+                            scratch, (size_t)SAGE_STATIC_SCRATCH_BYTES, status, stream);
 }

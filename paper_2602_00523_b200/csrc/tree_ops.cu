@@ -340,6 +340,7 @@ extern "C" const char* sage_status_string(int code) {
         case SAGE_ERR_UNSUPPORTED: return "outside the supported envelope";
         case SAGE_ERR_WORKSPACE: return "workspace missing or too small";
         case SAGE_ERR_CUDA: return "CUDA call failed";
+        case SAGE_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array holds";
         case SAGE_STATUS_BAD_TREE: return "device: parent array or node count violates the tree rules";
         case SAGE_STATUS_BAD_PAGE: return "device: page id out of range or sequence longer than its page table";
         case SAGE_STATUS_TIMEOUT: return "device: bounded wait expired";

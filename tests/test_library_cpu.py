@@ -25,7 +25,7 @@ def test_every_declared_symbol_is_exported():
 
 
 def test_status_strings():
-    for code in (0, 1, 2, 3, 4, 101, 102, 103, 104):
+    for code in (0, 1, 2, 3, 4, 5, 101, 102, 103, 104):
         assert sage.status_string(code) != "unknown status"
     assert sage.status_string(999) == "unknown status"
 
