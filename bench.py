@@ -374,7 +374,15 @@ def run_cuda(args):
         ach_tf = flops / (attn_ms * 1e-3) / 1e12
         ach_gb = kv_bytes / (attn_ms * 1e-3) / 1e9
         h2d = draft_host[0].numel() * 4 * 2 + q_host.numel() * 2 + tree_kv_host.numel() * 2
-        sample_s, full_s = oracle_sample_seconds(rows_sample=N_NODES, heads_sample=HKV)
+        if args.no_cpu_baseline:
+            cpu_baseline = None
+        else:
+            sample_s, full_s = oracle_sample_seconds(rows_sample=N_NODES, heads_sample=HKV)
+            cpu_baseline = {"value": 1.0 / full_s, "unit": "rounds/s", "cores": len(os.sched_getaffinity(0)),
+                            "kind": "oracle",
+                            "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
+                                      f"rows), attention, acceptance and compaction of 1 of the {N_LAYERS} layers; "
+                                      "the other layers are extrapolated"}
         n_splits_gt1 = sage.sage_tree_attention_workspace_size(N_LAYERS, 1, N_NODES, HQ, HKV, D, used_pages) > 16
         launches = 3 + 2 + (2 if n_splits_gt1 else 1) + 2 + 1 + 2
         line = {
@@ -382,22 +390,18 @@ def run_cuda(args):
             "warmup": args.warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "parallelism": f"replicas x{world}",
-                       "l2": "inputs larger than L2: 5.4 GB of K/V streamed per step"},
+                       "l2": f"inputs larger than L2: {kv_bytes / 1e9:.2f} GB of K/V streamed per step"},
             "e2e": {"value": e2e_value, "unit": "rounds/s", "h2d_bytes_per_step": int(h2d),
                     "d2h_bytes_per_step": int(result_host.numel() * 4), "ms_per_step": e2e_ms / steps},
             "gpu_launches": launches * steps,
             "clocks": clocks,
-            "roofline": {"kernel": "tree_attention (80 stacked layers per launch)", "bound": "tensor",
+            "roofline": {"kernel": f"tree_attention ({N_LAYERS} stacked layers per launch)", "bound": "tensor",
                          "achieved": ach_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": ach_tf / peaks["bf16_tflops_sustained"], "traffic": None,
                          "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
                          "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": ach_gb / peaks["hbm_gbs"]}},
-            "cpu_baseline": {"value": 1.0 / full_s, "unit": "rounds/s", "cores": len(os.sched_getaffinity(0)),
-                             "kind": "oracle",
-                             "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
-                                       "rows), attention, acceptance and compaction of 1 of the 80 layers; the other "
-                                       "79 layers are extrapolated"},
+            "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
     if world > 1:
@@ -405,12 +409,20 @@ def run_cuda(args):
 
 
 def main():
+    global N_LAYERS, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--layers", type=int, default=N_LAYERS,
+                    help="stacked layers per round (the workload has 80; fewer only for small profiler captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true",
+                    help="skip timing the CPU oracle (profiler captures)")
     args = ap.parse_args()
+    if args.layers != N_LAYERS:
+        WORKLOAD = WORKLOAD.replace(f"{N_LAYERS} layers", f"{args.layers} layers (reduced: not the benchmark workload)")
+        N_LAYERS = args.layers
     if args.impl == "reference":
         run_reference(args)
     else:
