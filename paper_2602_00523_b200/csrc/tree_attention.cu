@@ -5,7 +5,8 @@
 // form M = N*G query rows (<= 512).  A CTA owns up to two 128-row tiles of them and
 // one slice of the context (split-K).  The pipeline step is one 64-token page:
 //   TMA      : K and V pages -> 128B-swizzled shared memory, two 5-page rings, mbarriers
-//   tcgen05  : S_t = Q_t K^T (128 x 64, fp32) into TMEM, one elected thread issues
+//   tcgen05  : S_t = Q_t K^T (128 x 64, fp32) into TMEM; one warp per row tile issues, through
+//              one elected lane, with warp-uniform descriptor arithmetic
 //   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S, online
 //              softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back into TMEM
 //   tcgen05  : O_t += P_t V with P as the TMEM A operand, V MN-major from shared memory
@@ -29,7 +30,7 @@ constexpr int kPageBytes = kPageSize * kHeadDim * 2;        // one (page, head) 
 constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // one 64-wide d-half of a page: 8 KB
 constexpr int kQTileBytes = kRowTile * kHeadDim * 2;        // 32 KB
 constexpr int kQHalfBytes = kRowTile * 64 * 2;              // one 64-wide d-half of a Q tile: 16 KB
-constexpr int kAttnThreads = 320;              // 2 softmax warpgroups + TMA warp + MMA warp
+constexpr int kAttnThreads = 352;              // 2 softmax warpgroups + TMA warp + one MMA warp per row tile
 constexpr int kSmemBytes = 2 * kQTileBytes + 2 * kStages * kPageBytes + 1024 /*align*/ + 512 /*barriers*/;
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: far beyond any legitimate wait
 
@@ -54,7 +55,7 @@ struct __align__(8) Barriers {
     uint64_t s_full[2][2];     // [row tile][page parity]: scores of a page are in TMEM
     uint64_t p_full[2][2];     // [row tile][page parity]: probabilities of a page are in TMEM
     uint64_t pv_done[2];       // [row tile]: completes once per page, when its P V product has finished
-    uint64_t o_full;
+    uint64_t o_full[2];        // [row tile]: every MMA of the tile has finished
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -105,20 +106,32 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
 // ---- tcgen05 --------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+// One lane of a converged warp; the same lane every time for a full mask.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e != 0;
+}
+// The helpers below are called by a whole converged warp so that their operands stay warp-uniform;
+// only the `leader` lane executes the instruction.
+__device__ __forceinline__ void tc_commit(bool leader, uint64_t* bar) {
+    if (leader)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+template <bool kAcc>
+__device__ __forceinline__ void mma_ss(bool leader, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    if (leader)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(kAcc ? 1 : 0) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+__device__ __forceinline__ void mma_ts(bool leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    if (leader)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (quadrant*32 + i)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -245,14 +258,14 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     // ---- set-up: barriers, TMEM, Q tiles
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
-            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
-            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], n_rtiles);   // one release per MMA warp
+            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], n_rtiles);
         }
         for (int t = 0; t < 2; ++t) {
             for (int x = 0; x < 2; ++x) { mbar_init(&bars->s_full[t][x], 1); mbar_init(&bars->p_full[t][x], 4); }
             mbar_init(&bars->pv_done[t], 1);
+            mbar_init(&bars->o_full[t], 1);
         }
-        mbar_init(&bars->o_full, 1);
         bars->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -313,41 +326,48 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 }
             }
         }
-    } else if (warp == 9) {
-        // =========================== MMA issuer ===========================
-        const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-        auto issue_qk = [&](int t, int x, int slot) {
-            // S_t,x = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ss(tmem + t * 128 + x * 64,
-                       make_desc(q_addr + t * kQTileBytes + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
-                       make_desc(k_addr + slot * kPageBytes + (ks >> 2) * kPageHalfBytes + (ks & 3) * 32, 16, 1024),
-                       kIdescQK, ks > 0);
-        };
-        auto issue_pv = [&](int t, int x, int slot, bool first) {
-            // O_t += P_t,x V: 4 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + x * 64 + ks * 8,
-                       make_desc(v_addr + slot * kPageBytes + ks * 2048, kPageHalfBytes, 1024), kIdescPV,
-                       (!first || ks > 0));
-        };
+    } else if (warp >= 9) {
+        // =========================== MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1 ===========================
+        const int t = warp - 9;
+        const bool leader = elect_one();
         // lane 0 polls, the result is broadcast so that the warp never diverges on a wait
         auto wait_all = [&](uint64_t* bar, uint32_t parity) {
             int r = 1;
             if (lane == 0) r = mbar_wait(bar, parity, bars, p.status) ? 1 : 0;
             return __shfl_sync(0xffffffffu, r, 0) != 0;
         };
-        bool ok = ns > 0;
+        // descriptors differ only in their 14-bit start-address field (bytes >> 4); shared memory ends below 256 KB
+        const uint64_t dq = make_desc(smem_u32(sQ) + t * kQTileBytes, 16, 1024);
+        const uint64_t dk = make_desc(smem_u32(sK), 16, 1024);
+        const uint64_t dv = make_desc(smem_u32(sV), kPageHalfBytes, 1024);
+        const uint32_t s_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
+        auto issue_qk = [&](int x, int slot) {
+            // S_t,x = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
+            const uint64_t dks = dk + (uint64_t)((slot * kPageBytes) >> 4);
+            const uint32_t d = s_tmem + x * 64;
+            mma_ss<false>(leader, d, dq, dks, kIdescQK);
+#pragma unroll
+            for (int ks = 1; ks < 8; ++ks)
+                mma_ss<true>(leader, d, dq + (uint64_t)(((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4),
+                             dks + (uint64_t)(((ks >> 2) * kPageHalfBytes + (ks & 3) * 32) >> 4), kIdescQK);
+        };
+        auto issue_pv = [&](int x, int slot, bool first) {
+            // O_t += P_t,x V: 4 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
+            const uint64_t dvs = dv + (uint64_t)((slot * kPageBytes) >> 4);
+            const uint32_t a = s_tmem + x * 64;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ts(leader, o_tmem, a + ks * 8, dvs + (uint64_t)((ks * 2048) >> 4), kIdescPV, (!first || ks > 0) ? 1u : 0u);
+        };
+        bool ok = ns > 0 && t < n_rtiles;
         // prologue: scores of the first two pages
         for (int j = 0; ok && j < min(2, ns); ++j) {
             ok = wait_all(&bars->k_full[j], 0);
             if (!ok) break;
             tc_fence_after();
-            if (lane == 0) {
-                for (int t = 0; t < n_rtiles; ++t) { issue_qk(t, j, j); tc_commit(&bars->s_full[t][j]); }
-                tc_commit(&bars->k_empty[j]);
-            }
-            __syncwarp();
+            issue_qk(j, j);
+            tc_commit(leader, &bars->s_full[t][j]);
+            tc_commit(leader, &bars->k_empty[j]);
         }
         for (int j = 0; ok && j < ns; ++j) {
             const int x = j & 1, vslot = j % kStages;
@@ -356,6 +376,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             const int valid = min(kPageSize, T - (pg_begin + j) * kPageSize);
             if (valid < kPageSize) {
                 // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
+                // (both MMA warps write the same zeros; each orders its own writes before its own MMAs)
                 uint8_t* vb = sV + vslot * kPageBytes;
                 for (int c = lane; c < (kPageSize - valid) * 16; c += 32) {
                     const int r = valid + c / 16, ch = c % 16;
@@ -364,33 +385,24 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
+            ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(x, vslot, j == 0);
+            tc_commit(leader, &bars->pv_done[t]);
+            tc_commit(leader, &bars->v_empty[vslot]);
             const int jn = j + 2, kslot = jn % kStages;
-            for (int t = 0; ok && t < n_rtiles; ++t) {
-                ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
+            if (jn < ns) {
+                // the scores of page j+2 reuse this S buffer: in pipe order after P V of page j
+                ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
                 if (!ok) break;
                 tc_fence_after();
-                if (lane == 0) {
-                    issue_pv(t, x, vslot, j == 0);
-                    tc_commit(&bars->pv_done[t]);
-                    if (t == n_rtiles - 1) tc_commit(&bars->v_empty[vslot]);
-                }
-                if (jn < ns) {
-                    // the scores of page j+2 reuse this S buffer: in pipe order after P V of page j
-                    if (t == 0) {
-                        ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
-                        if (!ok) break;
-                        tc_fence_after();
-                    }
-                    if (lane == 0) {
-                        issue_qk(t, x, kslot);
-                        tc_commit(&bars->s_full[t][x]);
-                        if (t == n_rtiles - 1) tc_commit(&bars->k_empty[kslot]);
-                    }
-                }
-                __syncwarp();
+                issue_qk(x, kslot);
+                tc_commit(leader, &bars->s_full[t][x]);
+                tc_commit(leader, &bars->k_empty[kslot]);
             }
         }
-        if (lane == 0) tc_commit(&bars->o_full);      // arrives when every MMA above has completed
+        if (t < n_rtiles) tc_commit(leader, &bars->o_full[t]);     // arrives when every MMA of this tile has completed
         __syncwarp();
     } else {
         // =========================== softmax warpgroups ===========================
@@ -485,7 +497,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         }
         // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
         if (t < n_rtiles) {
-            if (ns > 0 && ok) ok = mbar_wait(&bars->o_full, 0, bars, p.status);
+            if (ns > 0 && ok) ok = mbar_wait(&bars->o_full[t], 0, bars, p.status);
             if (ok) tc_fence_after();
             const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
             const size_t row = (size_t)(n0 + node) * p.Hq + g * p.G + (row_ok ? R % p.G : 0);
