@@ -328,7 +328,14 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         }
     } else if (warp >= 9) {
         // =========================== MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1 ===========================
-        const int t = warp - 9;
+        // Broadcasts from lane 0 tell the compiler that these values are warp-uniform, so that the
+        // descriptor arithmetic and the loop control below can stay in the uniform datapath.
+        const int t = __shfl_sync(0xffffffffu, warp - 9, 0);
+        const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
+        const int ns = __shfl_sync(0xffffffffu, max(0, pg_end - pg_begin), 0);
+        const int n_rtiles = __shfl_sync(0xffffffffu, (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1, 0);
+        const int first_pos = __shfl_sync(0xffffffffu, pg_begin * kPageSize, 0);
+        const int T = __shfl_sync(0xffffffffu, L + N, 0);
         const bool leader = elect_one();
         // lane 0 polls, the result is broadcast so that the warp never diverges on a wait
         auto wait_all = [&](uint64_t* bar, uint32_t parity) {
@@ -373,7 +380,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             const int x = j & 1, vslot = j % kStages;
             ok = wait_all(&bars->v_full[vslot], (j / kStages) & 1);
             if (!ok) break;
-            const int valid = min(kPageSize, T - (pg_begin + j) * kPageSize);
+            const int valid = min(kPageSize, T - first_pos - j * kPageSize);
             if (valid < kPageSize) {
                 // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
                 // (both MMA warps write the same zeros; each orders its own writes before its own MMAs)
