@@ -59,6 +59,7 @@ struct __align__(8) Barriers {
     uint64_t p_full[2][2];     // [row tile][key half]: probabilities of a half step are in TMEM
     uint64_t pv_done[2];       // [row tile]: completes once per half step, when its P V product has finished
     uint64_t o_full[2];        // [row tile]: every MMA of the tile has finished
+    uint64_t turn[2];          // [row tile]: the other tile's warpgroup has finished a softmax step
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -192,6 +193,82 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// ---- packed fp32 pairs (one instruction works on two values) ----
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 2^x for a pair of x <= ~8 on the FMA and integer pipes instead of the special-function unit
+// (which delivers only 16 results per clock per SM and would otherwise bound the softmax):
+// x = n + f with n = round(x), f in [-0.5, 0.5]; 2^f by a cubic fitted to 7.5e-5 relative error
+// (well below the 2^-9 rounding of the bf16 probabilities); n goes straight into the exponent bits.
+// Inputs are clamped at -125, so that 2^x never leaves the normal range; -inf does not come here.
+__device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float& p0, float& p1) {
+    constexpr float kMagic = 12582912.f;             // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    float x0, x1;
+    f2_unpack(x2, x0, x1);
+    x2 = f2_pack(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t2 = f2_add(x2, f2_pack(kMagic, kMagic));
+    const uint64_t n2 = f2_add(t2, f2_pack(-kMagic, -kMagic));
+    const uint64_t f2 = f2_fma(n2, f2_pack(-1.f, -1.f), x2);
+    uint64_t q2 = f2_fma(f2, f2_pack(0.0551716685f, 0.0551716685f), f2_pack(0.2426111251f, 0.2426111251f));
+    q2 = f2_fma(q2, f2, f2_pack(0.6932609677f, 0.6932609677f));
+    q2 = f2_fma(q2, f2, f2_pack(0.9999280572f, 0.9999280572f));
+    float t0, t1, q0, q1;
+    f2_unpack(t2, t0, t1);
+    f2_unpack(q2, q0, q1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+// One 64-key half of a softmax step for one query row: p = 2^(s * scale + neg_ref), packed to
+// bf16 pairs, and their fp32 sum.  kEmu of every 8 column pairs take the FMA-pipe exp2.
+template <int kEmu>
+__device__ __forceinline__ float softmax_half(const uint32_t (&sr)[2][32], float scale, float neg_ref,
+                                              uint32_t (&pk)[32]) {
+    const uint64_t scale2 = f2_pack(scale, scale), nref2 = f2_pack(neg_ref, neg_ref);
+    uint64_t acc_a = f2_pack(0.f, 0.f), acc_b = acc_a;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const uint64_t s2 = f2_pack(__uint_as_float(sr[i >> 4][2 * (i & 15)]), __uint_as_float(sr[i >> 4][2 * (i & 15) + 1]));
+        const uint64_t x2 = f2_fma(s2, scale2, nref2);
+        float p0, p1;
+        if ((i & 7) < kEmu) {
+            exp2_pair_fma(x2, p0, p1);
+        } else {
+            float x0, x1;
+            f2_unpack(x2, x0, x1);
+            p0 = fast_exp2(x0);
+            p1 = fast_exp2(x1);
+        }
+        if (i & 1) acc_b = f2_add(acc_b, f2_pack(p0, p1));
+        else acc_a = f2_add(acc_a, f2_pack(p0, p1));
+        pk[i] = pack_bf16(p0, p1);
+    }
+    float a, b;
+    f2_unpack(f2_add(acc_a, acc_b), a, b);
+    return a + b;
+}
+
+#ifndef SAGE_EXP2_FMA_PAIRS
+#define SAGE_EXP2_FMA_PAIRS 3       // of every 8 column pairs
+#endif
+
 __global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ uint8_t smem_raw[];
@@ -264,6 +341,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             mbar_init(&bars->p_full[t][1], 4);
             mbar_init(&bars->pv_done[t], 1);
             mbar_init(&bars->o_full[t], 1);
+            mbar_init(&bars->turn[t], 4);
         }
         bars->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -427,6 +505,13 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         for (int j = 0; ok && j < nt; ++j) {
             ok = mbar_wait(&bars->s_full[t], j & 1, bars, p.status);
             if (!ok) break;
+            // The two warpgroups take turns (tile 0 step j, tile 1 step j, tile 0 step j+1, ...): a softmax
+            // step then has the special-function unit to itself and the tensor pipe serves the other tile
+            // meanwhile, instead of both tiles doing the same thing at the same time.
+            if (n_rtiles == 2 && (t == 1 || j > 0)) {
+                ok = mbar_wait(&bars->turn[t], (t == 1 ? j : j - 1) & 1, bars, p.status);
+                if (!ok) break;
+            }
             tc_fence_after();
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -484,25 +569,19 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                         tmem_st32(o_taddr + c * 32, orr);
                     }
                 }
-                float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * i]), p.scale_log2, neg_ref));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c][2 * i + 1]), p.scale_log2, neg_ref));
-                        sum0 += p0;
-                        sum1 += p1;
-                        pk[i] = pack_bf16(p0, p1);
-                    }
-                    tmem_st16(s_taddr + h * 64 + c * 16, pk);   // P (bf16 pairs) over the first 32 columns of this half of S
-                }
-                l_sum = l_sum * alpha + (sum0 + sum1);
+                uint32_t pk[32];
+                float sum;
+                if (pos0 + 64 > L) sum = softmax_half<0>(sr, p.scale_log2, neg_ref, pk);     // may hold -inf
+                else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref, pk);
+                tmem_st32(s_taddr + h * 64, pk);            // P (bf16 pairs) over the first 32 columns of this half of S
+                l_sum = l_sum * alpha + sum;
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->p_full[t][h]);
+                if (lane == 0) {
+                    mbar_arrive(&bars->p_full[t][h]);
+                    if (h == 1 && n_rtiles == 2) mbar_arrive(&bars->turn[t ^ 1]);
+                }
             }
         }
         // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
