@@ -237,32 +237,57 @@ __device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float& p0, float& p1)
 }
 
 // One 64-key half of a softmax step for one query row: p = 2^(s * scale + neg_ref), packed to
-// bf16 pairs, and their fp32 sum.  kEmu of every 8 column pairs take the FMA-pipe exp2.
+// bf16 pairs (in place, over the first 32 words of `sr`), and their fp32 sum.  kEmu of every 8
+// column pairs take the FMA-pipe exp2.  Written in stages over the whole row so that neighbouring
+// instructions are independent: a softmax warp mostly runs alone on its scheduler.
 template <int kEmu>
-__device__ __forceinline__ float softmax_half(const uint32_t (&sr)[2][32], float scale, float neg_ref,
-                                              uint32_t (&pk)[32]) {
+__device__ __forceinline__ float softmax_half(uint32_t (&sr)[64], float scale, float neg_ref) {
     const uint64_t scale2 = f2_pack(scale, scale), nref2 = f2_pack(neg_ref, neg_ref);
-    uint64_t acc_a = f2_pack(0.f, 0.f), acc_b = acc_a;
+    uint64_t x2[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        x2[i] = f2_fma(f2_pack(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), scale2, nref2);
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        const uint64_t s2 = f2_pack(__uint_as_float(sr[i >> 4][2 * (i & 15)]), __uint_as_float(sr[i >> 4][2 * (i & 15) + 1]));
-        const uint64_t x2 = f2_fma(s2, scale2, nref2);
         float p0, p1;
         if ((i & 7) < kEmu) {
-            exp2_pair_fma(x2, p0, p1);
+            exp2_pair_fma(x2[i], p0, p1);
         } else {
             float x0, x1;
-            f2_unpack(x2, x0, x1);
+            f2_unpack(x2[i], x0, x1);
             p0 = fast_exp2(x0);
             p1 = fast_exp2(x1);
         }
-        if (i & 1) acc_b = f2_add(acc_b, f2_pack(p0, p1));
-        else acc_a = f2_add(acc_a, f2_pack(p0, p1));
-        pk[i] = pack_bf16(p0, p1);
+        x2[i] = f2_pack(p0, p1);
+    }
+    uint64_t acc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = x2[i];
+#pragma unroll
+    for (int i = 4; i < 32; ++i) acc[i & 3] = f2_add(acc[i & 3], x2[i]);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        float p0, p1;
+        f2_unpack(x2[i], p0, p1);
+        sr[i] = pack_bf16(p0, p1);
     }
     float a, b;
-    f2_unpack(f2_add(acc_a, acc_b), a, b);
+    f2_unpack(f2_add(f2_add(acc[0], acc[1]), f2_add(acc[2], acc[3])), a, b);
     return a + b;
+}
+
+// O row *= alpha for the 32 rows of this warp (rare: only when a row maximum grew by more than 2^8).
+__device__ __noinline__ void rescale_o_rows(uint32_t o_taddr, float alpha) {
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+        uint32_t orr[32];
+        tmem_ld32(o_taddr + c * 32, orr);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+        tmem_st32(o_taddr + c * 32, orr);
+    }
+    tmem_wait_st();
 }
 
 #ifndef SAGE_EXP2_FMA_PAIRS
@@ -513,36 +538,33 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 if (!ok) break;
             }
             tc_fence_after();
-#pragma unroll
+#pragma unroll 1
             for (int h = 0; h < 2; ++h) {
-                uint32_t sr[2][32];
-                tmem_ld32(s_taddr + h * 64, sr[0]);
-                tmem_ld32(s_taddr + h * 64 + 32, sr[1]);
+                uint32_t sr[64];
+                tmem_ld32(s_taddr + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                tmem_ld32(s_taddr + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                 tmem_wait_ld();
                 const int pos0 = (t_begin + j) * kTileKeys + h * 64;
-                if (pos0 + 64 > L) {
+                const bool masked = pos0 + 64 > L;
+                if (masked) {
                     // reaches into the tree part (or past the end): apply the ancestor mask
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int jt = pos0 + c * 32 + i - L;        // tree slot; < 0 = prefix
-                            const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
-                            if (!vis) sr[c][i] = 0xff800000u;             // -inf
-                        }
+                    for (int i = 0; i < 64; ++i) {
+                        const int jt = pos0 + i - L;                  // tree slot; < 0 = prefix
+                        const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
+                        if (!vis) sr[i] = 0xff800000u;                // -inf
+                    }
                 }
-                // row max: four independent chains of three-input max
-                float mx4[4];
+                // row max: eight independent chains of three-input max
+                float mx8[8];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    float mq = __uint_as_float(sr[q4 >> 1][(q4 & 1) * 16]);
-#pragma unroll
-                    for (int i = 1; i < 15; i += 2)
-                        mq = max3(mq, __uint_as_float(sr[q4 >> 1][(q4 & 1) * 16 + i]),
-                                  __uint_as_float(sr[q4 >> 1][(q4 & 1) * 16 + i + 1]));
-                    mx4[q4] = fmaxf(mq, __uint_as_float(sr[q4 >> 1][(q4 & 1) * 16 + 15]));
+                for (int q8 = 0; q8 < 8; ++q8) {
+                    float mq = max3(__uint_as_float(sr[q8 * 8]), __uint_as_float(sr[q8 * 8 + 1]), __uint_as_float(sr[q8 * 8 + 2]));
+                    mq = max3(mq, __uint_as_float(sr[q8 * 8 + 3]), __uint_as_float(sr[q8 * 8 + 4]));
+                    mq = max3(mq, __uint_as_float(sr[q8 * 8 + 5]), __uint_as_float(sr[q8 * 8 + 6]));
+                    mx8[q8] = fmaxf(mq, __uint_as_float(sr[q8 * 8 + 7]));
                 }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), fmaxf(max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
                 const float m_cand = mx * p.scale_log2;
                 // lazy rescale: move the reference only when the row max grew by more than 2^8
                 const bool grow = m_cand > m_ref + 8.0f;
@@ -559,21 +581,12 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t orr[32];
-                        tmem_ld32(o_taddr + c * 32, orr);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                        tmem_st32(o_taddr + c * 32, orr);
-                    }
+                    rescale_o_rows(o_taddr, alpha);
                 }
-                uint32_t pk[32];
                 float sum;
-                if (pos0 + 64 > L) sum = softmax_half<0>(sr, p.scale_log2, neg_ref, pk);     // may hold -inf
-                else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref, pk);
-                tmem_st32(s_taddr + h * 64, pk);            // P (bf16 pairs) over the first 32 columns of this half of S
+                if (masked) sum = softmax_half<0>(sr, p.scale_log2, neg_ref);     // may hold -inf
+                else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref);
+                tmem_st32(s_taddr + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));   // P over the first 32 columns of this half of S
                 l_sum = l_sum * alpha + sum;
                 tmem_wait_st();
                 tc_fence_before();
