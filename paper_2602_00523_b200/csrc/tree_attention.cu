@@ -3,20 +3,17 @@
 //
 // Flash-decoding layout.  The N tree nodes x G query heads that share one KV head
 // form M = N*G query rows (<= 512).  A CTA owns up to two 128-row tiles of them and
-// one slice of the context (split-K).  The pipeline step is 128 keys (two 64-token pages):
-//   TMA      : K and V pages -> 128B-swizzled shared memory, 5-slot ring (K0 V0 K1 V1 ...), mbarriers
-//   tcgen05  : S_t = Q_t K^T (128 x 128, fp32) into TMEM; one warp per row tile issues, through
-//              one elected lane, with warp-uniform descriptor arithmetic.  (A 128 x 64 MMA
-//              occupies the tensor pipe as long as a 128 x 128 one, so scores are never
-//              computed in narrower pieces.)
-//   softmax  : one warpgroup per row tile, one thread per row, in two halves of 64 keys:
-//              tcgen05.ld S, online softmax in fp32 (log2 domain, lazy rescale), P -> bf16
-//              back into TMEM, so that P V of the first half runs under the second half
+// one slice of the context (split-K).  The pipeline step is one 64-token page:
+//   TMA      : K and V pages -> 128B-swizzled shared memory, two 5-page rings, mbarriers
+//   tcgen05  : S_t = Q_t K^T (128 x 64, fp32) into TMEM; one warp per row tile issues, through
+//              one elected lane, with warp-uniform descriptor arithmetic
+//   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S, online
+//              softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back into TMEM
 //   tcgen05  : O_t += P_t V with P as the TMEM A operand, V MN-major from shared memory
-// The two row tiles alternate: while one warpgroup does its softmax the tensor pipe works
-// for the other tile.
-// TMEM map (512 columns): S_t [128t, 128t+128) (P of key half h overlays columns
-// [128t+64h, 128t+64h+32)) and O_t [256+128t, 384+128t).
+// Every row tile has two S buffers (even / odd pages), so the tensor pipe computes the
+// scores of page j+1 while the warpgroup is busy with page j and never waits for it.
+// TMEM map (512 columns): tile t owns S_t,even [128t, 128t+64), S_t,odd [128t+64, 128t+128)
+// (P overlays the first 32 columns of its S buffer) and O_t [256+128t, 384+128t).
 // Slices are merged by attention_merge_kernel (warp per output row).  All waits are
 // bounded: on expiry the CTA records SAGE_STATUS_TIMEOUT, drains its copies, frees its
 // TMEM and returns.
@@ -26,16 +23,15 @@
 
 namespace sage {
 
-constexpr int kTileKeys = 128;                 // keys per pipeline step (two pages)
 constexpr int kRowTile = 128;                  // query rows per MMA tile
 constexpr int kRowsPerCta = 2 * kRowTile;
-constexpr int kSlots = 5;                      // K/V ring: K0 V0 K1 V1 K2 ...
-constexpr int kSlotBytes = kTileKeys * kHeadDim * 2;        // 32 KB
-constexpr int kHalfBytes = kTileKeys * 64 * 2;              // one 64-wide d-half of a tile: 16 KB
+constexpr int kStages = 5;                     // depth of the K ring and of the V ring, in pages
+constexpr int kPageBytes = kPageSize * kHeadDim * 2;        // one (page, head) tile: 16 KB
 constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // one 64-wide d-half of a page: 8 KB
 constexpr int kQTileBytes = kRowTile * kHeadDim * 2;        // 32 KB
+constexpr int kQHalfBytes = kRowTile * 64 * 2;              // one 64-wide d-half of a Q tile: 16 KB
 constexpr int kAttnThreads = 352;              // 2 softmax warpgroups + TMA warp + one MMA warp per row tile
-constexpr int kSmemBytes = 2 * kQTileBytes + kSlots * kSlotBytes + 1024 /*align*/ + 512 /*barriers*/;
+constexpr int kSmemBytes = 2 * kQTileBytes + 2 * kStages * kPageBytes + 1024 /*align*/ + 512 /*barriers*/;
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: far beyond any legitimate wait
 
 struct AttnParams {
@@ -54,12 +50,12 @@ struct AttnParams {
 };
 
 struct __align__(8) Barriers {
-    uint64_t full[kSlots], empty[kSlots];
-    uint64_t s_full[2];        // [row tile]: scores of a step are in TMEM
-    uint64_t p_full[2][2];     // [row tile][key half]: probabilities of a half step are in TMEM
-    uint64_t pv_done[2];       // [row tile]: completes once per half step, when its P V product has finished
+    uint64_t k_full[kStages], k_empty[kStages];
+    uint64_t v_full[kStages], v_empty[kStages];
+    uint64_t s_full[2][2];     // [row tile][page parity]: scores of a page are in TMEM
+    uint64_t p_full[2][2];     // [row tile][page parity]: probabilities of a page are in TMEM
+    uint64_t pv_done[2];       // [row tile]: completes once per page, when its P V product has finished
     uint64_t o_full[2];        // [row tile]: every MMA of the tile has finished
-    uint64_t turn[2];          // [row tile]: the other tile's warpgroup has finished a softmax step
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -182,10 +178,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
            ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = 128.
-constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescQK = kIdescBase;                    // A, B both K-major
-constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);       // B (= V) MN-major
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N as given.
+constexpr uint32_t idesc_f16(uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+constexpr uint32_t kIdescQK = idesc_f16(kPageSize);              // S (128 x 64): A, B both K-major
+constexpr uint32_t kIdescPV = idesc_f16(kHeadDim) | (1u << 16);  // O (128 x 128): B (= V) MN-major
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -302,8 +300,9 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     // 1024-byte alignment: the 128B swizzle pattern repeats every 1024 bytes of address
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                 // [2 tiles][2 d-halves][128 rows][128 B]
-    uint8_t* sKV = smem + 2 * kQTileBytes;              // [kSlots][2 d-halves][128 keys][128 B]
-    Barriers* bars = reinterpret_cast<Barriers*>(sKV + kSlots * kSlotBytes);
+    uint8_t* sK = smem + 2 * kQTileBytes;               // [kStages][2 d-halves][64 keys][128 B]
+    uint8_t* sV = sK + kStages * kPageBytes;            // [kStages][2 d-halves][64 keys][128 B]
+    Barriers* bars = reinterpret_cast<Barriers*>(sV + kStages * kPageBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x, rpair = blockIdx.y;
@@ -339,16 +338,16 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         }
         s_anc[tid] = a;
     }
-    // this CTA's slice of the context, in 128-key tiles
+    // this CTA's slice of the context, in pages
     const int n_pages_seq = (T + kPageSize - 1) / kPageSize;
-    const int n_tiles = (T + kTileKeys - 1) / kTileKeys;
-    const int per_split = (n_tiles + p.n_splits - 1) / p.n_splits;
-    const int t_begin = split * per_split;
-    const int t_end = min(n_tiles, t_begin + per_split);
-    const int nt = max(0, t_end - t_begin);             // pipeline steps
+    const int per_split = (n_pages_seq + p.n_splits - 1) / p.n_splits;
+    const int pg_begin = split * per_split;
+    const int pg_end = min(n_pages_seq, pg_begin + per_split);
+    const int ns = max(0, pg_end - pg_begin);           // pipeline steps
+    const int32_t* pages = p.page_table + (size_t)b * p.max_pages + pg_begin;
     // page ids of this slice must be valid before the TMA warp uses them as coordinates
-    for (int pg = t_begin * 2 + tid; pg < min(t_end * 2, n_pages_seq); pg += kAttnThreads) {
-        const int id = p.page_table[(size_t)b * p.max_pages + pg];
+    for (int j = tid; j < ns; j += kAttnThreads) {
+        const int id = pages[j];
         if (id < 0 || id >= p.n_pages) s_flag = 2;
     }
     __syncthreads();
@@ -359,14 +358,14 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 
     // ---- set-up: barriers, TMEM, Q tiles
     if (tid == 0) {
-        for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], n_rtiles); }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], n_rtiles);   // one release per MMA warp
+            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], n_rtiles);
+        }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(&bars->s_full[t], 1);
-            mbar_init(&bars->p_full[t][0], 4);
-            mbar_init(&bars->p_full[t][1], 4);
+            for (int x = 0; x < 2; ++x) { mbar_init(&bars->s_full[t][x], 1); mbar_init(&bars->p_full[t][x], 4); }
             mbar_init(&bars->pv_done[t], 1);
             mbar_init(&bars->o_full[t], 1);
-            mbar_init(&bars->turn[t], 4);
         }
         bars->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -387,40 +386,44 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 v = *reinterpret_cast<const uint4*>(p.q + row * kHeadDim + ch * 8);
             }
             const int half = ch >> 3, cc = ch & 7;
-            *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+            *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kQHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA unit
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
 
     if (warp == 8) {
         // =========================== TMA producer ===========================
         if (lane == 0) {
-            int issued = 0;
-            for (int n = 0; n < 2 * nt; ++n) {
-                const int slot = n % kSlots, use = n / kSlots;
-                if (use > 0 && !mbar_wait(&bars->empty[slot], (use - 1) & 1, bars, p.status)) break;
-                const int tile = t_begin + (n >> 1);
-                const CUtensorMap* map = (n & 1) ? &vmap : &kmap;
-                const int pg0 = tile * 2;
-                const int n_pg = min(2, n_pages_seq - pg0);
-                mbar_expect_tx(&bars->full[slot], (uint32_t)n_pg * 2 * kPageHalfBytes);
-                const uint32_t dst = smem_u32(sKV + slot * kSlotBytes);
-                for (int pp = 0; pp < n_pg; ++pp) {
-                    const int id = p.page_table[(size_t)b * p.max_pages + pg0 + pp];
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_4d(dst + h * kHalfBytes + pp * kPageHalfBytes, map, h * 64, 0, id * p.Hkv + g, layer,
-                                    &bars->full[slot]);
-                }
-                issued = n + 1;
+            int issued_k = 0, issued_v = 0;
+            for (int j = 0; j < ns; ++j) {
+                const int slot = j % kStages, use = j / kStages;
+                const int c2 = pages[j] * p.Hkv + g;
+                if (use > 0 && !mbar_wait(&bars->k_empty[slot], (use - 1) & 1, bars, p.status)) break;
+                mbar_expect_tx(&bars->k_full[slot], kPageBytes);
+                for (int h = 0; h < 2; ++h)
+                    tma_load_4d(smem_u32(sK + slot * kPageBytes + h * kPageHalfBytes), &kmap, h * 64, 0, c2, layer,
+                                &bars->k_full[slot]);
+                issued_k = j + 1;
+                if (use > 0 && !mbar_wait(&bars->v_empty[slot], (use - 1) & 1, bars, p.status)) break;
+                mbar_expect_tx(&bars->v_full[slot], kPageBytes);
+                for (int h = 0; h < 2; ++h)
+                    tma_load_4d(smem_u32(sV + slot * kPageBytes + h * kPageHalfBytes), &vmap, h * 64, 0, c2, layer,
+                                &bars->v_full[slot]);
+                issued_v = j + 1;
             }
             if (bars->abort) {
                 // drain: every issued copy must land before the CTA may exit
-                for (int n = max(0, issued - kSlots); n < issued; ++n) {
+                for (int n = max(0, issued_k - kStages); n < issued_k; ++n) {
                     const long long t0 = clock64();
-                    while (!mbar_try(&bars->full[n % kSlots], (n / kSlots) & 1) && clock64() - t0 < kWaitCycles) {}
+                    while (!mbar_try(&bars->k_full[n % kStages], (n / kStages) & 1) && clock64() - t0 < kWaitCycles) {}
+                }
+                for (int n = max(0, issued_v - kStages); n < issued_v; ++n) {
+                    const long long t0 = clock64();
+                    while (!mbar_try(&bars->v_full[n % kStages], (n / kStages) & 1) && clock64() - t0 < kWaitCycles) {}
                 }
             }
         }
@@ -430,10 +433,10 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         // descriptor arithmetic and the loop control below can stay in the uniform datapath.
         const int t = __shfl_sync(0xffffffffu, warp - 9, 0);
         const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
-        const int nt_u = __shfl_sync(0xffffffffu, nt, 0);
-        const int n_rt = __shfl_sync(0xffffffffu, n_rtiles, 0);
-        const int key0 = __shfl_sync(0xffffffffu, t_begin * kTileKeys, 0);
-        const int T_u = __shfl_sync(0xffffffffu, T, 0);
+        const int ns = __shfl_sync(0xffffffffu, max(0, pg_end - pg_begin), 0);
+        const int n_rtiles = __shfl_sync(0xffffffffu, (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1, 0);
+        const int first_pos = __shfl_sync(0xffffffffu, pg_begin * kPageSize, 0);
+        const int T = __shfl_sync(0xffffffffu, L + N, 0);
         const bool leader = elect_one();
         // lane 0 polls, the result is broadcast so that the warp never diverges on a wait
         auto wait_all = [&](uint64_t* bar, uint32_t parity) {
@@ -443,79 +446,74 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         };
         // descriptors differ only in their 14-bit start-address field (bytes >> 4); shared memory ends below 256 KB
         const uint64_t dq = make_desc(smem_u32(sQ) + t * kQTileBytes, 16, 1024);
-        const uint64_t dk = make_desc(smem_u32(sKV), 16, 1024);
-        const uint64_t dv = make_desc(smem_u32(sKV), kHalfBytes, 1024);
+        const uint64_t dk = make_desc(smem_u32(sK), 16, 1024);
+        const uint64_t dv = make_desc(smem_u32(sV), kPageHalfBytes, 1024);
         const uint32_t s_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
-        auto issue_qk = [&](int slot) {
-            // S_t = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
-            const uint64_t dks = dk + (uint64_t)((slot * kSlotBytes) >> 4);
-            mma_ss<false>(leader, s_tmem, dq, dks, kIdescQK);
+        auto issue_qk = [&](int x, int slot) {
+            // S_t,x = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
+            const uint64_t dks = dk + (uint64_t)((slot * kPageBytes) >> 4);
+            const uint32_t d = s_tmem + x * 64;
+            mma_ss<false>(leader, d, dq, dks, kIdescQK);
 #pragma unroll
-            for (int ks = 1; ks < 8; ++ks) {
-                const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                mma_ss<true>(leader, s_tmem, dq + off, dks + off, kIdescQK);
-            }
+            for (int ks = 1; ks < 8; ++ks)
+                mma_ss<true>(leader, d, dq + (uint64_t)(((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4),
+                             dks + (uint64_t)(((ks >> 2) * kPageHalfBytes + (ks & 3) * 32) >> 4), kIdescQK);
         };
-        auto issue_pv = [&](int h, int slot, bool first) {
-            // O_t += P_t,h V_h: 4 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
-            const uint64_t dvs = dv + (uint64_t)((slot * kSlotBytes + h * kPageHalfBytes) >> 4);
-            const uint32_t a = s_tmem + h * 64;
+        auto issue_pv = [&](int x, int slot, bool first) {
+            // O_t += P_t,x V: 4 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
+            const uint64_t dvs = dv + (uint64_t)((slot * kPageBytes) >> 4);
+            const uint32_t a = s_tmem + x * 64;
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
                 mma_ts(leader, o_tmem, a + ks * 8, dvs + (uint64_t)((ks * 2048) >> 4), kIdescPV, (!first || ks > 0) ? 1u : 0u);
         };
-        bool ok = nt_u > 0 && t < n_rt;
-        if (ok) ok = wait_all(&bars->full[0], 0);
-        if (ok) {
-            tc_fence_after();
-            issue_qk(0);
-            tc_commit(leader, &bars->s_full[t]);
-            tc_commit(leader, &bars->empty[0]);
-        }
-        for (int j = 0; ok && j < nt_u; ++j) {
-            const int nv = 2 * j + 1, vslot = nv % kSlots;
-            ok = wait_all(&bars->full[vslot], (nv / kSlots) & 1);
+        bool ok = ns > 0 && t < n_rtiles;
+        // prologue: scores of the first two pages
+        for (int j = 0; ok && j < min(2, ns); ++j) {
+            ok = wait_all(&bars->k_full[j], 0);
             if (!ok) break;
-            const int valid = min(kTileKeys, T_u - key0 - j * kTileKeys);
-            if (valid < kTileKeys) {
+            tc_fence_after();
+            issue_qk(j, j);
+            tc_commit(leader, &bars->s_full[t][j]);
+            tc_commit(leader, &bars->k_empty[j]);
+        }
+        for (int j = 0; ok && j < ns; ++j) {
+            const int x = j & 1, vslot = j % kStages;
+            ok = wait_all(&bars->v_full[vslot], (j / kStages) & 1);
+            if (!ok) break;
+            const int valid = min(kPageSize, T - first_pos - j * kPageSize);
+            if (valid < kPageSize) {
                 // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
                 // (both MMA warps write the same zeros; each orders its own writes before its own MMAs)
-                uint8_t* vb = sKV + vslot * kSlotBytes;
-                for (int c = lane; c < (kTileKeys - valid) * 16; c += 32) {
+                uint8_t* vb = sV + vslot * kPageBytes;
+                for (int c = lane; c < (kPageSize - valid) * 16; c += 32) {
                     const int r = valid + c / 16, ch = c % 16;
-                    *reinterpret_cast<uint4*>(vb + (ch >> 3) * kHalfBytes + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(vb + (ch >> 3) * kPageHalfBytes + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
-            ok = wait_all(&bars->p_full[t][0], j & 1);
+            ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            issue_pv(0, vslot, j == 0);
+            issue_pv(x, vslot, j == 0);
             tc_commit(leader, &bars->pv_done[t]);
-            const int nk = 2 * (j + 1), kslot = nk % kSlots;
-            if (j + 1 < nt_u) {                               // off the critical path: the next K tile
-                ok = wait_all(&bars->full[kslot], (nk / kSlots) & 1);
+            tc_commit(leader, &bars->v_empty[vslot]);
+            const int jn = j + 2, kslot = jn % kStages;
+            if (jn < ns) {
+                // the scores of page j+2 reuse this S buffer: in pipe order after P V of page j
+                ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
                 if (!ok) break;
-            }
-            ok = wait_all(&bars->p_full[t][1], j & 1);
-            if (!ok) break;
-            tc_fence_after();
-            issue_pv(1, vslot, false);
-            tc_commit(leader, &bars->pv_done[t]);
-            tc_commit(leader, &bars->empty[vslot]);
-            if (j + 1 < nt_u) {
-                // the next scores overwrite S_t and both P halves: in pipe order after this step's P V
-                issue_qk(kslot);
-                tc_commit(leader, &bars->s_full[t]);
-                tc_commit(leader, &bars->empty[kslot]);
+                tc_fence_after();
+                issue_qk(x, kslot);
+                tc_commit(leader, &bars->s_full[t][x]);
+                tc_commit(leader, &bars->k_empty[kslot]);
             }
         }
-        if (t < n_rt) tc_commit(leader, &bars->o_full[t]);     // arrives when every MMA of this tile has completed
+        if (t < n_rtiles) tc_commit(leader, &bars->o_full[t]);     // arrives when every MMA of this tile has completed
         __syncwarp();
     } else {
         // =========================== softmax warpgroups ===========================
-        const uint32_t tmem = bars->tmem_base;
         const int t = warp >> 2;                        // row tile of this warpgroup
         const int r = tid & 127;                        // row inside the tile == TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -527,79 +525,66 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         const uint64_t anc = s_anc[node];
         float m_ref = -INFINITY, l_sum = 0.f;
         bool ok = (t < n_rtiles);
-        for (int j = 0; ok && j < nt; ++j) {
-            ok = mbar_wait(&bars->s_full[t], j & 1, bars, p.status);
+        for (int j = 0; ok && j < ns; ++j) {
+            const int x = j & 1;
+            ok = mbar_wait(&bars->s_full[t][x], (j >> 1) & 1, bars, p.status);
             if (!ok) break;
-            // The two warpgroups take turns (tile 0 step j, tile 1 step j, tile 0 step j+1, ...): a softmax
-            // step then has the special-function unit to itself and the tensor pipe serves the other tile
-            // meanwhile, instead of both tiles doing the same thing at the same time.
-            if (n_rtiles == 2 && (t == 1 || j > 0)) {
-                ok = mbar_wait(&bars->turn[t], (t == 1 ? j : j - 1) & 1, bars, p.status);
-                if (!ok) break;
-            }
             tc_fence_after();
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-                uint32_t sr[64];
-                tmem_ld32(s_taddr + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                tmem_ld32(s_taddr + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-                tmem_wait_ld();
-                const int pos0 = (t_begin + j) * kTileKeys + h * 64;
-                const bool masked = pos0 + 64 > L;
-                if (masked) {
-                    // reaches into the tree part (or past the end): apply the ancestor mask
+            uint32_t sr[64];
+            tmem_ld32(s_taddr + x * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+            tmem_ld32(s_taddr + x * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+            tmem_wait_ld();
+            const int pos0 = (pg_begin + j) * kPageSize;
+            const bool masked = pos0 + kPageSize > L;
+            if (masked) {
+                // page reaches into the tree part (or past the end): apply the ancestor mask
 #pragma unroll
-                    for (int i = 0; i < 64; ++i) {
-                        const int jt = pos0 + i - L;                  // tree slot; < 0 = prefix
-                        const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
-                        if (!vis) sr[i] = 0xff800000u;                // -inf
-                    }
-                }
-                // row max: eight independent chains of three-input max
-                float mx8[8];
-#pragma unroll
-                for (int q8 = 0; q8 < 8; ++q8) {
-                    float mq = max3(__uint_as_float(sr[q8 * 8]), __uint_as_float(sr[q8 * 8 + 1]), __uint_as_float(sr[q8 * 8 + 2]));
-                    mq = max3(mq, __uint_as_float(sr[q8 * 8 + 3]), __uint_as_float(sr[q8 * 8 + 4]));
-                    mq = max3(mq, __uint_as_float(sr[q8 * 8 + 5]), __uint_as_float(sr[q8 * 8 + 6]));
-                    mx8[q8] = fmaxf(mq, __uint_as_float(sr[q8 * 8 + 7]));
-                }
-                const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), fmaxf(max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-                const float m_cand = mx * p.scale_log2;
-                // lazy rescale: move the reference only when the row max grew by more than 2^8
-                const bool grow = m_cand > m_ref + 8.0f;
-                float alpha = 1.0f;
-                if (grow) {
-                    alpha = fast_exp2(m_ref - m_cand);          // 0 when m_ref was -inf
-                    m_ref = m_cand;
-                }
-                const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                const int hs = 2 * j + h;                       // half steps done so far
-                if (hs > 0 && __any_sync(0xffffffffu, grow)) {
-                    // O_t *= alpha, once the P V product of the previous half step has finished
-                    ok = mbar_wait(&bars->pv_done[t], (hs - 1) & 1, bars, p.status);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                    rescale_o_rows(o_taddr, alpha);
-                }
-                float sum;
-                if (masked) sum = softmax_half<0>(sr, p.scale_log2, neg_ref);     // may hold -inf
-                else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref);
-                tmem_st32(s_taddr + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));   // P over the first 32 columns of this half of S
-                l_sum = l_sum * alpha + sum;
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&bars->p_full[t][h]);
-                    if (h == 1 && n_rtiles == 2) mbar_arrive(&bars->turn[t ^ 1]);
+                for (int i = 0; i < 64; ++i) {
+                    const int jt = pos0 + i - L;                      // tree slot; < 0 = prefix
+                    const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
+                    if (!vis) sr[i] = 0xff800000u;                    // -inf
                 }
             }
+            // row max: eight independent chains of three-input max
+            float mx8[8];
+#pragma unroll
+            for (int q8 = 0; q8 < 8; ++q8) {
+                float mq = max3(__uint_as_float(sr[q8 * 8]), __uint_as_float(sr[q8 * 8 + 1]), __uint_as_float(sr[q8 * 8 + 2]));
+                mq = max3(mq, __uint_as_float(sr[q8 * 8 + 3]), __uint_as_float(sr[q8 * 8 + 4]));
+                mq = max3(mq, __uint_as_float(sr[q8 * 8 + 5]), __uint_as_float(sr[q8 * 8 + 6]));
+                mx8[q8] = fmaxf(mq, __uint_as_float(sr[q8 * 8 + 7]));
+            }
+            const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), fmaxf(max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+            const float m_cand = mx * p.scale_log2;
+            // lazy rescale: move the reference only when the row max grew by more than 2^8
+            const bool grow = m_cand > m_ref + 8.0f;
+            float alpha = 1.0f;
+            if (grow) {
+                alpha = fast_exp2(m_ref - m_cand);          // 0 when m_ref was -inf
+                m_ref = m_cand;
+            }
+            const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                // O_t *= alpha, once the P V product of page j-1 has finished
+                ok = mbar_wait(&bars->pv_done[t], (j - 1) & 1, bars, p.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                rescale_o_rows(o_taddr, alpha);
+            }
+            float sum;
+            if (masked) sum = softmax_half<0>(sr, p.scale_log2, neg_ref);     // may hold -inf
+            else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref);
+            tmem_st32(s_taddr + x * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));   // P over the first 32 columns of this S buffer
+            l_sum = l_sum * alpha + sum;
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->p_full[t][x]);
         }
         // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
         if (t < n_rtiles) {
-            if (nt > 0 && ok) ok = mbar_wait(&bars->o_full[t], 0, bars, p.status);
+            if (ns > 0 && ok) ok = mbar_wait(&bars->o_full[t], 0, bars, p.status);
             if (ok) tc_fence_after();
             const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
             const size_t row = (size_t)(n0 + node) * p.Hq + g * p.G + (row_ok ? R % p.G : 0);
@@ -611,12 +596,12 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             } else {
                 const size_t pr = ((size_t)layer * p.n_splits + split) * rows_total + row;
                 po = p.part_o + pr * kHeadDim;
-                if (row_ok && ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = (nt > 0) ? l_sum : 0.f; }
+                if (row_ok && ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = (ns > 0) ? l_sum : 0.f; }
             }
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t orr[32];
-                if (nt > 0 && ok) {
+                if (ns > 0 && ok) {
                     tmem_ld32(o_taddr + c * 32, orr);
                     tmem_wait_ld();
                 } else {
@@ -649,7 +634,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     __syncthreads();
     if (warp == 9) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(bars->tmem_base), "r"(512) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     }
 }
 
@@ -693,11 +678,10 @@ __global__ void attention_merge_kernel(AttnParams p) {
 
 static int pick_splits(int n_layers, int batch, int n_kv_heads, int G, int max_pages) {
     // One CTA is resident per SM.  Take the smallest slice count whose CTA count fills whole
-    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 4 key tiles per slice.
+    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 8 pages per slice.
     const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
     const long base = (long)n_layers * batch * n_kv_heads * row_pairs;
-    const int tiles = (max_pages + 1) / 2;
-    int s_max = tiles / 4;
+    int s_max = max_pages / 8;
     if (s_max > 32) s_max = 32;
     if (s_max < 1) s_max = 1;
     int best = 1;
