@@ -289,7 +289,7 @@ __device__ __noinline__ void rescale_o_rows(uint32_t o_taddr, float alpha) {
 }
 
 #ifndef SAGE_EXP2_FMA_PAIRS
-#define SAGE_EXP2_FMA_PAIRS 3       // of every 8 column pairs
+#define SAGE_EXP2_FMA_PAIRS 1       // of every 8 column pairs (measured best with both warpgroups busy at once)
 #endif
 
 __global__ void __launch_bounds__(kAttnThreads, 1)

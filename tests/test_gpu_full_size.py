@@ -1,0 +1,97 @@
+"""GPU parity at the benchmark's full size and launch configuration: 80 stacked layers,
+16384-token prefix with a shuffled page table, 60-node tree, 64/8/128 heads.
+
+The fp64 oracle cannot redo 80 layers in test time, so three sampled layers are compared
+with it element by element (on the very bytes the GPU used), and properties that hold at
+any size cover the rest: every output finite, every layer of the compacted cache equal to
+the input except for the accepted rows, which must be copies of their source rows.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2602_00523_b200 as sage
+from helpers import check_attention, dev_i32, host_bits
+from workloads import make_template
+from workloads.gen import _rng
+
+pytestmark = pytest.mark.gpu
+
+HQ, HKV, D, P = 64, 8, 128, 64
+N_LAYERS, L, N, N_VISUAL = 80, 16384, 60, 32 * 196
+SAMPLED_LAYERS = (0, 37, 79)
+
+
+def _build():
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(523000 + 4000 + 77)
+    used = (L + N + P - 1) // P
+    n_pages = int(np.ceil(used * 1.125))
+    perm = _rng(4, 1).permutation(n_pages)[:used].astype(np.int32)
+    k = torch.empty((N_LAYERS, n_pages, HKV, P, D), dtype=torch.bfloat16, device=dev)
+    v = torch.empty_like(k)
+    vis = torch.from_numpy(perm[:N_VISUAL // P].astype(np.int64)).to(dev)
+    for pool in (k, v):
+        for layer in range(N_LAYERS):
+            pool[layer].normal_(generator=gen)
+            pool[layer, vis] *= 1.5
+    q = torch.empty((N_LAYERS, N, HQ, D), dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+    tree = make_template(3, 10, N)
+    return dict(k=k, v=v, q=q, perm=perm, tree=tree, page_table=dev_i32(perm.reshape(1, -1)),
+                seq_len=dev_i32([L]), parent=dev_i32(tree["parent"]), offs=dev_i32([0, N]))
+
+
+def test_attention_80_layers_sampled_layers_match_the_oracle_and_all_outputs_are_finite():
+    w = _build()
+    st = sage.new_status()
+    out = sage.sage_tree_attention(w["q"], w["k"], w["v"], w["page_table"], w["seq_len"], w["parent"], w["offs"],
+                                   1.0 / np.sqrt(D), status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0, sage.status_string(int(st.item()))
+    assert bool(torch.isfinite(out.float()).all())
+    # this launch must be the one the benchmark times: no split-K workspace
+    assert sage.sage_tree_attention_workspace_size(N_LAYERS, 1, N, HQ, HKV, D, w["page_table"].shape[1]) <= 16
+    offs = np.array([0, N], np.int32)
+    for layer in SAMPLED_LAYERS:
+        want = oracle.tree_attention(host_bits(w["q"][layer]), host_bits(w["k"][layer]), host_bits(w["v"][layer]),
+                                     w["perm"].reshape(1, -1), np.array([L], np.int32), w["tree"]["parent"], offs,
+                                     HQ, HKV, D, P, 1.0 / np.sqrt(D))
+        check_attention(host_bits(out[layer]), want)
+
+
+def test_compaction_80_layers_moves_exactly_the_accepted_rows():
+    w = _build()
+    k0, v0 = w["k"].clone(), w["v"].clone()
+    # a root path of the tree: from the root, always to the last child (far from its destination slot)
+    parent = w["tree"]["parent"]
+    path = [0]
+    while len(path) < 4:
+        kids = [i for i in range(N) if parent[i] == path[-1]]
+        if not kids:
+            break
+        path.append(kids[-1])
+    max_path = 9
+    path_arr = np.full((1, max_path), -1, np.int32)
+    path_arr[0, :len(path)] = path
+    st = sage.new_status()
+    seq = w["seq_len"].clone()
+    sage.sage_compact_kv(w["k"], w["v"], w["page_table"], seq, dev_i32(path_arr), dev_i32([len(path)]), status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and int(seq.item()) == L + len(path)
+    # sampled layers against the oracle, byte for byte
+    for layer in SAMPLED_LAYERS:
+        wk, wv, wl = oracle.compact_kv(host_bits(k0[layer:layer + 1]), host_bits(v0[layer:layer + 1]),
+                                       w["perm"].reshape(1, -1), np.array([L], np.int32), path_arr,
+                                       np.array([len(path)], np.int32), P)
+        assert np.array_equal(host_bits(w["k"][layer:layer + 1]), wk)
+        assert np.array_equal(host_bits(w["v"][layer:layer + 1]), wv)
+        assert int(wl[0]) == L + len(path)
+    # every layer: destination rows are copies of their sources, nothing else changed
+    for new, old in ((w["k"], k0), (w["v"], v0)):
+        expect = old.clone()
+        for j, node in enumerate(path):
+            src, dst = L + node, L + j
+            expect[:, int(w["perm"][dst // P]), :, dst % P, :] = old[:, int(w["perm"][src // P]), :, src % P, :]
+        assert torch.equal(new.view(torch.int16), expect.view(torch.int16))
