@@ -181,6 +181,18 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------
 # CUDA path
 # ----------------------------------------------------------------------------------------------
+def max_over_ranks(value, world, device):
+    """The slowest rank's device time: every rank runs an independent replica of the round (the
+    path has no exchange step), so the job's time is the maximum."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -348,10 +360,7 @@ def run_cuda(args):
         clocks = sampler.stop(t0, t1)
         ms = e0.elapsed_time(e1)
         attn_ms = float(np.mean([a.elapsed_time(b) for a, b in attn_events]))
-        if world > 1:
-            tt = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
+        ms = max_over_ranks(ms, world, dev)
         return ms, attn_ms, clocks, seen
 
     ms, attn_ms, clocks, _ = timed(False)
