@@ -43,6 +43,14 @@ WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefi
            "page 64 shuffled, 60-node tree, 80 layers, logits 60x152064 fp32"
 
 
+# DRAM bytes per layer of the attention launch, from the ncu counter capture of the current
+# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 619.14 MB over 9 layers,
+# profiles/tree_attention_kernel_config4_9layers.md).  Traffic grows in proportion to the layer
+# count (every layer streams its own K/V once).  Set to None whenever the kernel changes until the
+# counters are taken again.
+ATTN_DRAM_BYTES_PER_LAYER = 619.14e6 / 9
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -406,7 +414,10 @@ def run_cuda(args):
             "clocks": clocks,
             "roofline": {"kernel": f"tree_attention ({N_LAYERS} stacked layers per launch)", "bound": "tensor",
                          "achieved": ach_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": ach_tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                         "frac": ach_tf / peaks["bf16_tflops_sustained"],
+                         "traffic": None if ATTN_DRAM_BYTES_PER_LAYER is None else ATTN_DRAM_BYTES_PER_LAYER * N_LAYERS,
+                         "traffic_unit": "bytes per launch (ncu DRAM read+write on a 9-layer capture, scaled by layers)",
+                         "algorithmic_bytes": kv_bytes,
                          "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
                          "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": ach_gb / peaks["hbm_gbs"]}},
