@@ -56,6 +56,7 @@ struct __align__(8) Barriers {
     uint64_t p_full[2][2];     // [row tile][page parity]: probabilities of a page are in TMEM
     uint64_t pv_done[2];       // [row tile]: completes once per page, when its P V product has finished
     uint64_t o_full[2];        // [row tile]: every MMA of the tile has finished
+    uint64_t q_ready;          // the query tiles are staged in shared memory
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -367,6 +368,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             mbar_init(&bars->pv_done[t], 1);
             mbar_init(&bars->o_full[t], 1);
         }
+        mbar_init(&bars->q_ready, 8);
         bars->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -375,6 +377,10 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                      ::"r"(smem_u32(&bars->tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // From here the TMA producer streams K/V while the softmax warps stage the query tiles.
     if (warp < 8) {
         // Q rows -> K-major 128B-swizzled tiles; rows past M are zero
         for (int c = tid; c < n_rtiles * kRowTile * 16; c += 256) {
@@ -389,10 +395,9 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kQHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA unit
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->q_ready);
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
     if (warp == 8) {
@@ -468,6 +473,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 mma_ts(leader, o_tmem, a + ks * 8, dvs + (uint64_t)((ks * 2048) >> 4), kIdescPV, (!first || ks > 0) ? 1u : 0u);
         };
         bool ok = ns > 0 && t < n_rtiles;
+        if (ok) ok = wait_all(&bars->q_ready, 0);
         // prologue: scores of the first two pages
         for (int j = 0; ok && j < min(2, ns); ++j) {
             ok = wait_all(&bars->k_full[j], 0);
