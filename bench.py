@@ -371,7 +371,31 @@ def run_cuda(args):
         ms = max_over_ranks(ms, world, dev)
         return ms, attn_ms, clocks, seen
 
+    def per_layer_attention_us(passes=3):
+        """Attention launched layer by layer, as a model's forward does (other layers' work would sit
+        in between): 80 single-layer calls walk over the 80 layers' K/V (5.5 GB), so no layer's K/V is
+        still in L2 when its turn comes.  Returns the mean microseconds per call (split-K + merge)."""
+        tree_parent = bank_parent[1, :N_NODES].contiguous()
+        ws1 = torch.empty(max(16, sage.sage_tree_attention_workspace_size(1, 1, N_NODES, HQ, HKV, D, used_pages)),
+                          dtype=torch.uint8, device=dev)
+
+        def sweep():
+            for layer in range(N_LAYERS):
+                sage.sage_tree_attention(q_dev[layer:layer + 1], k_pool[layer:layer + 1], v_pool[layer:layer + 1],
+                                         page_table, seq_len, tree_parent, node_offsets, 1.0 / np.sqrt(D),
+                                         out=attn_out[layer:layer + 1], ws=ws1, status=status)
+        sweep()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(passes):
+            sweep()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)
+
     ms, attn_ms, clocks, _ = timed(False)
+    layer_us = per_layer_attention_us()
     if int(status.item()) != 0:
         raise RuntimeError("device status: " + sage.status_string(int(status.item())))
     e2e_ms, _, _, seen = timed(True)
@@ -421,6 +445,10 @@ def run_cuda(args):
                          "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
                          "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": ach_gb / peaks["hbm_gbs"]}},
+            "attention_per_layer": {"us_per_call": layer_us, "tflops": flops / N_LAYERS / (layer_us * 1e-6) / 1e12,
+                                    "gbs": kv_bytes / N_LAYERS / (layer_us * 1e-6) / 1e9,
+                                    "note": "80 single-layer calls walking over all layers' K/V (split-K + merge "
+                                            "kernels, launch gaps included)"},
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

@@ -382,17 +382,28 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     tc_fence_after();
     // From here the TMA producer streams K/V while the softmax warps stage the query tiles.
     if (warp < 8) {
-        // Q rows -> K-major 128B-swizzled tiles; rows past M are zero
-        for (int c = tid; c < n_rtiles * kRowTile * 16; c += 256) {
-            const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
-            const int R = rpair * kRowsPerCta + t * kRowTile + r;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (R < M) {
-                const size_t row = ((size_t)layer * p.sum_nodes + n0 + R / p.G) * p.Hq + g * p.G + R % p.G;
-                v = *reinterpret_cast<const uint4*>(p.q + row * kHeadDim + ch * 8);
+        // Q rows -> K-major 128B-swizzled tiles; rows past M are zero.  Eight 16-byte loads are in
+        // flight per thread before the first store (the loads are latency-bound otherwise).
+        for (int c0 = tid; c0 < n_rtiles * kRowTile * 16; c0 += 256 * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * 256;
+                const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
+                const int R = rpair * kRowsPerCta + t * kRowTile + r;
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (R < M) {
+                    const size_t row = ((size_t)layer * p.sum_nodes + n0 + R / p.G) * p.Hq + g * p.G + R % p.G;
+                    v[u] = *reinterpret_cast<const uint4*>(p.q + row * kHeadDim + ch * 8);
+                }
             }
-            const int half = ch >> 3, cc = ch & 7;
-            *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kQHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * 256;
+                const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
+                const int half = ch >> 3, cc = ch & 7;
+                *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kQHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v[u];
+            }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA unit
         __syncwarp();
