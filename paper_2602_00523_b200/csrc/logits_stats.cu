@@ -87,31 +87,42 @@ __global__ void __launch_bounds__(kPartialThreads) logits_partial_kernel(Partial
     // 16-byte loads: `begin` and row_stride are multiples of 4 elements.
     const int n4 = (end - begin) >> 2;
     const float4* src4 = reinterpret_cast<const float4*>(rowp + begin);
-    for (int i0 = 0; i0 < n4; i0 += kPartialThreads) {
-        const int i = i0 + tid;
-        const bool live = i < n4;
-        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-        if (live) v = __ldcs(src4 + i);
-        if (live) {
-            const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
-            if (m4 > m) {
-                const float c = expf(m - m4);
-                t = c * fmaf(m - m4, s, t);
-                s *= c;
-                m = m4;
-            }
-            const float d0 = v.x - m, d1 = v.y - m, d2 = v.z - m, d3 = v.w - m;
-            const float e0 = expf(d0), e1 = expf(d1), e2 = expf(d2), e3 = expf(d3);
-            s += (e0 + e1) + (e2 + e3);
-            t += fmaf(d0, e0, d1 * e1) + fmaf(d2, e2, d3 * e3);
+    // Four 16-byte loads are in flight per thread before the first is used: the chunk is short
+    // (a few dozen elements per thread), so the pass is bound by load latency, not by bandwidth.
+    for (int i0 = 0; i0 < n4; i0 += 4 * kPartialThreads) {
+        float4 vv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * kPartialThreads + tid;
+            vv[u] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            if (i < n4) vv[u] = __ldcs(src4 + i);
         }
-        const bool hit = live && (v.x >= wq.thr || v.y >= wq.thr || v.z >= wq.thr || v.w >= wq.thr);
-        if (__any_sync(0xffffffffu, hit)) {
-            const int base = begin + 4 * i;
-            wq.offer(live && v.x >= wq.thr, v.x, base + 0, lane);
-            wq.offer(live && v.y >= wq.thr, v.y, base + 1, lane);
-            wq.offer(live && v.z >= wq.thr, v.z, base + 2, lane);
-            wq.offer(live && v.w >= wq.thr, v.w, base + 3, lane);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * kPartialThreads + tid;
+            const bool live = i < n4;
+            const float4 v = vv[u];
+            if (live) {
+                const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+                if (m4 > m) {
+                    const float c = expf(m - m4);
+                    t = c * fmaf(m - m4, s, t);
+                    s *= c;
+                    m = m4;
+                }
+                const float d0 = v.x - m, d1 = v.y - m, d2 = v.z - m, d3 = v.w - m;
+                const float e0 = expf(d0), e1 = expf(d1), e2 = expf(d2), e3 = expf(d3);
+                s += (e0 + e1) + (e2 + e3);
+                t += fmaf(d0, e0, d1 * e1) + fmaf(d2, e2, d3 * e3);
+            }
+            const bool hit = live && (v.x >= wq.thr || v.y >= wq.thr || v.z >= wq.thr || v.w >= wq.thr);
+            if (__any_sync(0xffffffffu, hit)) {
+                const int base = begin + 4 * i;
+                wq.offer(live && v.x >= wq.thr, v.x, base + 0, lane);
+                wq.offer(live && v.y >= wq.thr, v.y, base + 1, lane);
+                wq.offer(live && v.z >= wq.thr, v.z, base + 2, lane);
+                wq.offer(live && v.w >= wq.thr, v.w, base + 3, lane);
+            }
         }
     }
     // ragged tail of the last chunk (vocab % 4 elements)
