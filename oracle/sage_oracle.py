@@ -267,3 +267,55 @@ def compact_kv(k_pool, v_pool, page_table, seq_len, path, path_len, page_size):
             v_new[:, dp, :, ds, :] = v_pool[:, sp, :, ss, :]
         new_len[b] = L + int(path_len[b])
     return k_new, v_new, new_len
+
+
+# --------------------------------------------------------------------------
+# Dynamic tree construction, one level at a time  (Section 3.2: "Hierarchical
+# Width Decay", Eq. 12, and "Dynamic Tree Construction").  A path is in the tree
+# iff at every level l its rank p_l < W_l and its cumulative probability exceeds
+# theta_l = 0.1 * l / D(alpha); W_1 = W(alpha), and beyond the first level
+# W_l = W(alpha) / l * (0.5 + P_parent).  Readings taken where the paper is
+# silent: P_parent is the cumulative path probability of the parent (1 for the
+# root); "p_l < W_l" is used as it stands with the real-valued W_l (no rounding
+# rule is invented); a level l exists iff l <= D(alpha); nodes are added in
+# breadth-first order (parents by index, ranks ascending) until N_max nodes.
+# Decisions are taken in fp64 on the fp32 inputs; cumulative log-probabilities
+# are fp32 sums (the library does the same).  "parity unpinned" for these
+# readings; the level-wise construction itself is pinned against the path rule
+# evaluated directly on every path of a full k-ary tree.
+# --------------------------------------------------------------------------
+def grow_tree_level(parent, rank, depth, token, cum_logprob, n_nodes, frontier_begin,
+                    topk_idx, topk_logprob, alpha, n_max=64,
+                    d_min=3.0, d_max=8.0, w_min=2.0, w_max=10.0):
+    """Adds the next level to one tree (arrays of capacity >= n_max, modified in place).
+
+    Nodes frontier_begin .. n_nodes-1 are the deepest level so far; row i of topk_idx /
+    topk_logprob holds node i's k best next tokens and their log-probabilities (descending).
+    Returns (new n_nodes, new frontier_begin)."""
+    a = float(np.float32(alpha))
+    D = d_min + a * (d_max - d_min)
+    W = w_min + (1.0 - a) * (w_max - w_min)
+    k = topk_idx.shape[1]
+    n = int(n_nodes)
+    if n <= int(frontier_begin):
+        return n, int(frontier_begin)
+    level = int(depth[int(frontier_begin)]) + 1
+    new_begin = n
+    if float(level) > D:
+        return n, new_begin
+    theta = 0.1 * level / D
+    for u in range(int(frontier_begin), int(n_nodes)):
+        p_parent = float(np.exp(np.float64(cum_logprob[u])))
+        w_l = W if level == 1 else W / level * (0.5 + p_parent)
+        for r in range(k):
+            if not (float(r) < w_l):
+                break
+            c = np.float32(np.float32(cum_logprob[u]) + np.float32(topk_logprob[u, r]))
+            if not (float(np.exp(np.float64(c))) > theta):
+                break
+            if n >= n_max:
+                return n, new_begin
+            parent[n], rank[n], depth[n] = u, r, level
+            token[n], cum_logprob[n] = topk_idx[u, r], c
+            n += 1
+    return n, new_begin
