@@ -145,6 +145,30 @@ int sage_select_tree(const float *alpha, const int32_t *alpha_row, int batch,
                      int32_t *next_parent, int32_t *next_rank, int32_t *next_node_offsets,
                      int32_t *status, void *stream);
 
+/* Dynamic tree construction, one level per call (Section 3.2: "Hierarchical Width Decay", Eq. 12,
+ * and "Dynamic Tree Construction"; Algorithm 1, the tree update of phase 3).  Every sequence b owns
+ * SAGE_MAX_NODES node slots: slot b*SAGE_MAX_NODES + i holds node i (parent, rank among its parent's
+ * candidates, depth, token, cum_logprob = log of the cumulative path probability).  Nodes
+ * frontier_begin[b] .. n_nodes[b]-1 are the deepest level so far; row b*SAGE_MAX_NODES + i of
+ * topk_idx / topk_logprob ([.][k], log-probabilities descending, e.g. from sage_expand_topk on the
+ * draft model's logits of that node) holds node i's candidates; only frontier rows are read.
+ * The call appends level l = depth(frontier) + 1: with alpha = alpha[alpha_row ? alpha_row[b] : b],
+ * D = D(alpha), W = W(alpha) (Eq. 10, Eq. 11), W_1 = W and W_l = W / l * (0.5 + P_parent) beyond the
+ * first level (P_parent = cumulative probability of the parent, 1 for the root), candidate rank r of
+ * a frontier node joins iff r < W_l and its cumulative probability exceeds theta_l = 0.1 * l / D;
+ * the scan of a row stops at the first rank that fails.  No level beyond D is opened.  Children are
+ * appended in breadth-first order (parents by index, ranks ascending) until n_max nodes exist.
+ * Afterwards frontier_begin[b] is the first new node and n_nodes[b] the new count; a call that finds
+ * nothing to expand changes nothing.  The caller starts a tree with node 0 (parent -1, depth 0,
+ * cum_logprob 0, its token), n_nodes = 1, frontier_begin = 0.  `policy` is a host pointer (its
+ * thresholds are not used here).  Decisions are taken in fp64 on the fp32 inputs. */
+int sage_grow_tree(const int32_t *topk_idx, const float *topk_logprob, int k,
+                   const float *alpha, const int32_t *alpha_row, int batch,
+                   const sage_tree_policy *policy, int n_max,
+                   int32_t *parent, int32_t *rank, int32_t *depth, int32_t *token, float *cum_logprob,
+                   int32_t *n_nodes, int32_t *frontier_begin,
+                   int32_t *status, void *stream);
+
 /* Tree attention mask as per-node ancestor bitsets (Section 2.2: each token attends
  * only to its ancestors; Algorithm 1 TreeAttnMask).  anc[i] has bit j set iff j == i or
  * j is an ancestor of i (local indices).  sage_tree_attention builds the same bitsets

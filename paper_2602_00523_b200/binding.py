@@ -65,6 +65,9 @@ _lib.sage_expand_topk_static.argtypes = [_vp, _i, _i, _i64, _i, _i, _vp, _vp, _v
 _lib.sage_select_tree.restype = _i
 _lib.sage_select_tree.argtypes = [_vp, _vp, _i, ctypes.POINTER(SagePolicy), _vp, _vp, _vp,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sage_grow_tree.restype = _i
+_lib.sage_grow_tree.argtypes = [_vp, _vp, _i, _vp, _vp, _i, ctypes.POINTER(SagePolicy), _i,
+                                _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sage_build_ancestor_mask.restype = _i
 _lib.sage_build_ancestor_mask.argtypes = [_vp, _vp, _i, _vp, _vp, _vp]
 _lib.sage_tree_attention.restype = _i
@@ -199,6 +202,22 @@ def sage_select_tree(alpha: torch.Tensor, policy: SagePolicy, *, alpha_row=None,
                                  _ptr(o.get("next_node_offsets")), _ptr(status), _stream(stream))
     _check(code, "sage_select_tree")
     return o
+
+
+def sage_grow_tree(topk_idx: torch.Tensor, topk_logprob: torch.Tensor, alpha: torch.Tensor, policy: SagePolicy,
+                   tree: Dict[str, torch.Tensor], *, alpha_row=None, n_max: int = SAGE_MAX_NODES, status=None,
+                   stream=None) -> Dict[str, torch.Tensor]:
+    """One level of dynamic tree construction, in place on ``tree`` (parent, rank, depth, token:
+    int32 [batch * SAGE_MAX_NODES]; cum_logprob fp32 of the same length; n_nodes, frontier_begin:
+    int32 [batch]).  topk_idx / topk_logprob: [batch * SAGE_MAX_NODES, k]."""
+    batch = tree["n_nodes"].numel()
+    k = topk_idx.shape[1]
+    code = _lib.sage_grow_tree(_ptr(topk_idx), _ptr(topk_logprob), k, _ptr(alpha), _ptr(alpha_row), batch,
+                               ctypes.byref(policy), n_max, _ptr(tree["parent"]), _ptr(tree["rank"]),
+                               _ptr(tree["depth"]), _ptr(tree["token"]), _ptr(tree["cum_logprob"]),
+                               _ptr(tree["n_nodes"]), _ptr(tree["frontier_begin"]), _ptr(status), _stream(stream))
+    _check(code, "sage_grow_tree")
+    return tree
 
 
 def sage_build_ancestor_mask(parent: torch.Tensor, node_offsets: torch.Tensor, *, out=None, status=None, stream=None):

@@ -270,6 +270,91 @@ __global__ void advance_seq_len_kernel(int32_t* seq_len, const int32_t* path_len
     if (pl >= 0 && pl <= max_path) seq_len[b] += pl;
 }
 
+// ---------------------------------------------------------------------------
+// Dynamic tree construction, one level per launch (Section 3.2: hierarchical width
+// decay, Eq. 12, and "Dynamic Tree Construction").  One block per sequence, one
+// thread per frontier node.  A child of rank r of frontier node u joins the tree iff
+// r < W_l and exp(cum_logprob) > theta_l; both tests only ever cut a suffix of the
+// (descending) candidate row, so each node contributes a prefix of its ranks, and the
+// children are laid out in breadth-first order by a prefix sum.  Decisions are taken
+// in fp64 on the fp32 inputs; cumulative log-probabilities are fp32 sums.
+// ---------------------------------------------------------------------------
+struct GrowParams {
+    const int32_t* topk_idx;
+    const float* topk_logprob;
+    int k;
+    const float* alpha;
+    const int32_t* alpha_row;
+    sage_tree_policy pol;
+    int n_max;
+    int32_t *parent, *rank, *depth, *token;
+    float* cum_logprob;
+    int32_t *n_nodes, *frontier_begin;
+    int32_t* status;
+};
+
+__global__ void __launch_bounds__(SAGE_MAX_NODES) grow_tree_kernel(GrowParams p) {
+    __shared__ int s_count[SAGE_MAX_NODES];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int base = b * SAGE_MAX_NODES;
+    const int n = p.n_nodes[b], fb = p.frontier_begin[b];
+    if (n < 1 || n > p.n_max || fb < 0 || fb > n) {
+        if (tid == 0) report_status(p.status, SAGE_STATUS_BAD_TREE);
+        return;
+    }
+    if (fb == n) return;                                   // nothing left to expand
+    const int level = p.depth[base + fb] + 1;
+    const double a = (double)p.alpha[p.alpha_row ? p.alpha_row[b] : b];
+    // explicit roundings: no fused multiply-add, so that a host check in plain fp64 sees the same D and W
+    const double D = __dadd_rn((double)p.pol.d_min, __dmul_rn(a, (double)p.pol.d_max - (double)p.pol.d_min));
+    const double W = __dadd_rn((double)p.pol.w_min, __dmul_rn(1.0 - a, (double)p.pol.w_max - (double)p.pol.w_min));
+    if ((double)level > D) {                               // the tree has reached its depth
+        if (tid == 0) p.frontier_begin[b] = n;
+        return;
+    }
+    const double theta = 0.1 * (double)level / D;
+    const int node = fb + tid;
+    int count = 0;
+    float cum_u = 0.f;
+    if (node < n) {
+        cum_u = p.cum_logprob[base + node];
+        const double p_parent = exp((double)cum_u);
+        const double w_l = (level == 1) ? W : W / (double)level * (0.5 + p_parent);
+        const float* lp = p.topk_logprob + (size_t)(base + node) * p.k;
+        for (int r = 0; r < p.k; ++r) {
+            if (!((double)r < w_l)) break;
+            const float c = __fadd_rn(cum_u, lp[r]);
+            if (!(exp((double)c) > theta)) break;
+            ++count;
+        }
+    }
+    s_count[tid] = count;
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int i = 0; i < SAGE_MAX_NODES; ++i) {
+        const int c = s_count[i];
+        if (i < tid) before += c;
+        total += c;
+    }
+    if (node < n) {
+        const float* lp = p.topk_logprob + (size_t)(base + node) * p.k;
+        const int32_t* ix = p.topk_idx + (size_t)(base + node) * p.k;
+        for (int r = 0; r < count; ++r) {
+            const int pos = n + before + r;
+            if (pos >= p.n_max) break;                     // node budget: breadth-first prefix
+            p.parent[base + pos] = node;
+            p.rank[base + pos] = r;
+            p.depth[base + pos] = level;
+            p.token[base + pos] = ix[r];
+            p.cum_logprob[base + pos] = __fadd_rn(cum_u, lp[r]);
+        }
+    }
+    if (tid == 0) {
+        p.n_nodes[b] = min(n + total, p.n_max);
+        p.frontier_begin[b] = n;
+    }
+}
+
 }  // namespace sage
 
 using namespace sage;
@@ -330,6 +415,25 @@ extern "C" int sage_compact_kv(void* k_pool, void* v_pool, int64_t layer_stride_
                     max_pages_per_seq, batch, max_path, n_kv_heads, page_table, seq_len, path, path_len, status};
     compact_kv_kernel<<<dim3(batch, n_layers), 256, 0, as_stream(stream)>>>(p);
     advance_seq_len_kernel<<<(batch + 127) / 128, 128, 0, as_stream(stream)>>>(seq_len, path_len, batch, max_path);
+    return launch_status();
+}
+
+extern "C" int sage_grow_tree(const int32_t* topk_idx, const float* topk_logprob, int k, const float* alpha,
+                              const int32_t* alpha_row, int batch, const sage_tree_policy* policy, int n_max,
+                              int32_t* parent, int32_t* rank, int32_t* depth, int32_t* token, float* cum_logprob,
+                              int32_t* n_nodes, int32_t* frontier_begin, int32_t* status, void* stream) {
+    if (!topk_idx || !topk_logprob || !alpha || !policy || !parent || !rank || !depth || !token || !cum_logprob ||
+        !n_nodes || !frontier_begin)
+        return SAGE_ERR_INVALID_ARG;
+    if (batch < 0 || k < 1 || n_max < 1) return SAGE_ERR_INVALID_ARG;
+    if (k > SAGE_MAX_TOPK || n_max > SAGE_MAX_NODES) return SAGE_ERR_UNSUPPORTED;
+    if (!(policy->d_max >= policy->d_min) || !(policy->d_min > 0.f) || !(policy->w_max >= policy->w_min) ||
+        !(policy->w_min > 0.f))
+        return SAGE_ERR_INVALID_ARG;
+    if (batch == 0) return SAGE_OK;
+    GrowParams p{topk_idx, topk_logprob, k, alpha, alpha_row, *policy, n_max, parent, rank, depth, token,
+                 cum_logprob, n_nodes, frontier_begin, status};
+    grow_tree_kernel<<<batch, SAGE_MAX_NODES, 0, as_stream(stream)>>>(p);
     return launch_status();
 }
 

@@ -74,3 +74,18 @@ def test_host_side_argument_validation_needs_no_gpu():
     pol = sage.make_policy([0.5])
     assert lib.sage_select_tree(fake, None, 0, ctypes.byref(pol), fake, None, None, None, None, None, None, None,
                                 None, None, None) == sage.SAGE_OK      # empty batch: nothing to do
+
+
+def test_grow_tree_argument_validation_needs_no_gpu():
+    lib = sage.lib()
+    fake = ctypes.c_void_p(0x1000)
+    pol = sage.make_policy([])
+    args = [fake, fake, 10, fake, None, 1, ctypes.byref(pol), 64, fake, fake, fake, fake, fake, fake, fake, None, None]
+    bad = list(args); bad[2] = 17
+    assert lib.sage_grow_tree(*bad) == sage.SAGE_ERR_UNSUPPORTED
+    bad = list(args); bad[7] = 65
+    assert lib.sage_grow_tree(*bad) == sage.SAGE_ERR_UNSUPPORTED
+    bad = list(args); bad[0] = None
+    assert lib.sage_grow_tree(*bad) == sage.SAGE_ERR_INVALID_ARG
+    ok = list(args); ok[5] = 0
+    assert lib.sage_grow_tree(*ok) == sage.SAGE_OK
