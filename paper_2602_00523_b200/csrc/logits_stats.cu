@@ -36,6 +36,15 @@ __device__ __forceinline__ uint64_t make_key(float x, int idx) {
     return ((uint64_t)order_key(x) << 32) | (uint32_t)(0xffffffffu - (uint32_t)idx);
 }
 
+// e^d for d <= 0 through the hardware 2^x (relative error about 2^-22): one multiply and one
+// special-function instruction instead of the library routine's range reduction.  The moments
+// built from it are merged in fp64; the entropy stays well inside its 1e-5 bound.
+__device__ __forceinline__ float exp_neg(float d) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(d * 1.4426950408889634f));
+    return y;
+}
+
 struct WarpQueue {
     uint64_t q;        // lane j < K: j-th best key so far (0 = empty)
     uint64_t kth;      // key in lane K-1 (same in all lanes)
@@ -111,17 +120,22 @@ __global__ void __launch_bounds__(kPartialThreads) logits_partial_kernel(Partial
                     m = m4;
                 }
                 const float d0 = v.x - m, d1 = v.y - m, d2 = v.z - m, d3 = v.w - m;
-                const float e0 = expf(d0), e1 = expf(d1), e2 = expf(d2), e3 = expf(d3);
+                const float e0 = exp_neg(d0), e1 = exp_neg(d1), e2 = exp_neg(d2), e3 = exp_neg(d3);
                 s += (e0 + e1) + (e2 + e3);
                 t += fmaf(d0, e0, d1 * e1) + fmaf(d2, e2, d3 * e3);
             }
-            const bool hit = live && (v.x >= wq.thr || v.y >= wq.thr || v.z >= wq.thr || v.w >= wq.thr);
+            // A lane's largest component goes first: it lifts the queue's threshold, so that most of
+            // the other components no longer qualify (matters while the queue is still filling).
+            const float m4q = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+            const bool hit = live && m4q >= wq.thr;
             if (__any_sync(0xffffffffu, hit)) {
                 const int base = begin + 4 * i;
-                wq.offer(live && v.x >= wq.thr, v.x, base + 0, lane);
-                wq.offer(live && v.y >= wq.thr, v.y, base + 1, lane);
-                wq.offer(live && v.z >= wq.thr, v.z, base + 2, lane);
-                wq.offer(live && v.w >= wq.thr, v.w, base + 3, lane);
+                const int top = (v.x == m4q) ? 0 : (v.y == m4q) ? 1 : (v.z == m4q) ? 2 : 3;   // lowest index on ties
+                wq.offer(hit, m4q, base + top, lane);
+                wq.offer(live && top != 0 && v.x >= wq.thr, v.x, base + 0, lane);
+                wq.offer(live && top != 1 && v.y >= wq.thr, v.y, base + 1, lane);
+                wq.offer(live && top != 2 && v.z >= wq.thr, v.z, base + 2, lane);
+                wq.offer(live && top != 3 && v.w >= wq.thr, v.w, base + 3, lane);
             }
         }
     }
