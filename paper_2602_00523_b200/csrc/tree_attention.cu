@@ -540,12 +540,20 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         const bool row_ok = R < M;
         const int node = row_ok ? R / p.G : 0;
         const uint64_t anc = s_anc[node];
+        const bool warp_live = rpair * kRowsPerCta + t * kRowTile + (warp & 3) * 32 < M;
         float m_ref = -INFINITY, l_sum = 0.f;
         bool ok = (t < n_rtiles);
         for (int j = 0; ok && j < ns; ++j) {
             const int x = j & 1;
             ok = mbar_wait(&bars->s_full[t][x], (j >> 1) & 1, bars, p.status);
             if (!ok) break;
+            if (!warp_live) {
+                // none of this warp's 32 rows exists (ragged last tile): keep the barrier protocol
+                // going, leave the probabilities of these rows as they are; their outputs are never stored
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->p_full[t][x]);
+                continue;
+            }
             tc_fence_after();
             uint32_t sr[64];
             tmem_ld32(s_taddr + x * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
