@@ -44,11 +44,11 @@ WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefi
 
 
 # DRAM bytes per layer of the attention launch, from the ncu counter capture of the current
-# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 619.14 MB over 9 layers,
+# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 618.83 MB over 9 layers,
 # profiles/tree_attention_kernel_config4_9layers.md).  Traffic grows in proportion to the layer
 # count (every layer streams its own K/V once).  Set to None whenever the kernel changes until the
 # counters are taken again.
-ATTN_DRAM_BYTES_PER_LAYER = 619.14e6 / 9
+ATTN_DRAM_BYTES_PER_LAYER = 618.83e6 / 9
 
 
 def load_peaks():
@@ -395,7 +395,7 @@ def run_cuda(args):
         return e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)
 
     ms, attn_ms, clocks, _ = timed(False)
-    layer_us = per_layer_attention_us()
+    layer_us = None if args.no_per_layer else per_layer_attention_us()
     if int(status.item()) != 0:
         raise RuntimeError("device status: " + sage.status_string(int(status.item())))
     e2e_ms, _, _, seen = timed(True)
@@ -445,10 +445,11 @@ def run_cuda(args):
                          "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
                          "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": ach_gb / peaks["hbm_gbs"]}},
-            "attention_per_layer": {"us_per_call": layer_us, "tflops": flops / N_LAYERS / (layer_us * 1e-6) / 1e12,
-                                    "gbs": kv_bytes / N_LAYERS / (layer_us * 1e-6) / 1e9,
-                                    "note": "80 single-layer calls walking over all layers' K/V (split-K + merge "
-                                            "kernels, launch gaps included)"},
+            "attention_per_layer": None if layer_us is None else {
+                "us_per_call": layer_us, "tflops": flops / N_LAYERS / (layer_us * 1e-6) / 1e12,
+                "gbs": kv_bytes / N_LAYERS / (layer_us * 1e-6) / 1e9,
+                "note": "80 single-layer calls walking over all layers' K/V (split-K + merge kernels, launch "
+                        "gaps included)"},
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
@@ -465,6 +466,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=N_LAYERS,
                     help="stacked layers per round (the workload has 80; fewer only for small profiler captures)")
+    ap.add_argument("--no-per-layer", action="store_true",
+                    help="skip the layer-by-layer attention timing (profiler launch lists of the round alone)")
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip timing the CPU oracle (profiler captures)")
     args = ap.parse_args()
