@@ -510,18 +510,21 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
+            // the K page of step j+2 is normally there already: look now, while the softmax of page j
+            // is still running, instead of between the two MMA groups below
+            const int jn = j + 2, kslot = jn % kStages;
+            if (jn < ns) {
+                ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
+                if (!ok) break;
+            }
             ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
             issue_pv(x, vslot, j == 0);
             tc_commit(leader, &bars->pv_done[t]);
             tc_commit(leader, &bars->v_empty[vslot]);
-            const int jn = j + 2, kslot = jn % kStages;
             if (jn < ns) {
                 // the scores of page j+2 reuse this S buffer: in pipe order after P V of page j
-                ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
-                if (!ok) break;
-                tc_fence_after();
                 issue_qk(x, kslot);
                 tc_commit(leader, &bars->s_full[t][x]);
                 tc_commit(leader, &bars->k_empty[kslot]);
