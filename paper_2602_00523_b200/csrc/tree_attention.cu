@@ -494,10 +494,13 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             tc_commit(leader, &bars->s_full[t][j]);
             tc_commit(leader, &bars->k_empty[j]);
         }
-        for (int j = 0; ok && j < ns; ++j) {
-            const int x = j & 1, vslot = j % kStages;
-            ok = wait_all(&bars->v_full[vslot], (j / kStages) & 1);
-            if (!ok) break;
+        // The V page of step j and the K page of step j+2 are looked up one step ahead (`stage_inputs`),
+        // while the softmax of the previous page is still running, so that only the wait for the
+        // probabilities sits between the softmax and the MMAs that depend on it.
+        auto stage_inputs = [&](int j) -> bool {
+            if (j >= ns) return true;
+            const int vslot = j % kStages;
+            if (!wait_all(&bars->v_full[vslot], (j / kStages) & 1)) return false;
             const int valid = min(kPageSize, T - first_pos - j * kPageSize);
             if (valid < kPageSize) {
                 // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
@@ -510,13 +513,14 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
-            // the K page of step j+2 is normally there already: look now, while the softmax of page j
-            // is still running, instead of between the two MMA groups below
+            const int jn = j + 2;
+            if (jn < ns && !wait_all(&bars->k_full[jn % kStages], (jn / kStages) & 1)) return false;
+            return true;
+        };
+        if (ok) ok = stage_inputs(0);
+        for (int j = 0; ok && j < ns; ++j) {
+            const int x = j & 1, vslot = j % kStages;
             const int jn = j + 2, kslot = jn % kStages;
-            if (jn < ns) {
-                ok = wait_all(&bars->k_full[kslot], (jn / kStages) & 1);
-                if (!ok) break;
-            }
             ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
@@ -529,6 +533,7 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
                 tc_commit(leader, &bars->s_full[t][x]);
                 tc_commit(leader, &bars->k_empty[kslot]);
             }
+            ok = stage_inputs(j + 1);
         }
         if (t < n_rtiles) tc_commit(leader, &bars->o_full[t]);     // arrives when every MMA of this tile has completed
         __syncwarp();
