@@ -23,11 +23,15 @@ Pin status (what fixes each function other than itself, see tests/test_oracle_*)
   grow_tree_level    the path-inclusion rule evaluated directly on every path of a full
                      k-ary tree (tiny k, depth); its readings of the paper's rounding /
                      P_parent / stopping order are "parity unpinned"
+  update_history     hand-computed windows; its long-run behaviour under a simulated
+                     acceptance process whose mean is the closed form of Theorem 2
+                     (expected_acceptance_length, itself checked by simulation); step, clamps
+                     and the warm-up rule are "parity unpinned"
   Which row of a tree supplies the distribution that drives selection is not
   fixed by the paper: "parity unpinned" for that choice (the caller passes the
   row index to both sides).
 """
 from .sage_oracle import (  # noqa: F401
     ancestor_mask, tree_attention, softmax_entropy, topk, topk_logprob,
-    confidence, select_tree, expand_gather, accept, compact_kv, widen_bf16, grow_tree_level,
+    confidence, select_tree, expand_gather, accept, compact_kv, widen_bf16, grow_tree_level, update_history, expected_acceptance_length,
 )

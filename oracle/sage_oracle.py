@@ -319,3 +319,36 @@ def grow_tree_level(parent, rank, depth, token, cum_logprob, n_nodes, frontier_b
             token[n], cum_logprob[n] = topk_idx[u, r], c
             n += 1
     return n, new_begin
+
+
+# --------------------------------------------------------------------------
+# Adaptive history tracking  (Section 3.3 "Adaptive History Tracking"; window
+# size 10 and thresholds 2 / 3 in Section 5.1 "Implementation details").  A
+# sliding window of recent acceptance lengths tau; when their mean falls below
+# the lower threshold the maximum depth goes down, above the upper threshold it
+# goes up, in between it stays.  The paper gives neither the step nor the
+# clamps nor what happens before the window is full: here the step and the
+# clamp range are parameters, and nothing moves until `min_samples` values are
+# in the window ("parity unpinned" for those readings).
+# --------------------------------------------------------------------------
+def update_history(window_buf, count, d_max, tau, window=10, lower=2.0, upper=3.0, step=1.0,
+                   d_lo=3.0, d_hi=8.0, min_samples=10):
+    """One sequence: pushes tau into the ring `window_buf` (int32 [window], in place) and returns
+    (new count, new d_max)."""
+    window_buf[int(count) % window] = int(tau)
+    count = int(count) + 1
+    n = min(count, window)
+    d = float(np.float32(d_max))
+    if n >= min_samples:
+        mean = float(np.sum(window_buf[:n].astype(np.int64))) / n
+        if mean < lower:
+            d = max(float(d_lo), d - float(step))
+        elif mean > upper:
+            d = min(float(d_hi), d + float(step))
+    return count, np.float32(d)
+
+
+def expected_acceptance_length(p, gamma, depth):
+    """Closed form of Theorem 2 (Section 4.2): E[tau] = sum_{l=1..D} p^l gamma^(l(l-1)/2) for greedy-path
+    speculation whose level-l token is accepted with probability p gamma^(l-1)."""
+    return float(sum(p ** l * gamma ** (l * (l - 1) / 2.0) for l in range(1, int(depth) + 1)))
