@@ -161,13 +161,35 @@ int sage_select_tree(const float *alpha, const int32_t *alpha_row, int batch,
  * Afterwards frontier_begin[b] is the first new node and n_nodes[b] the new count; a call that finds
  * nothing to expand changes nothing.  The caller starts a tree with node 0 (parent -1, depth 0,
  * cum_logprob 0, its token), n_nodes = 1, frontier_begin = 0.  `policy` is a host pointer (its
- * thresholds are not used here).  Decisions are taken in fp64 on the fp32 inputs. */
+ * thresholds are not used here).  d_max_seq, when not NULL, gives every sequence its own maximum
+ * depth (e.g. from sage_update_history) in place of policy->d_max.  Decisions are taken in fp64 on
+ * the fp32 inputs. */
 int sage_grow_tree(const int32_t *topk_idx, const float *topk_logprob, int k,
                    const float *alpha, const int32_t *alpha_row, int batch,
                    const sage_tree_policy *policy, int n_max,
                    int32_t *parent, int32_t *rank, int32_t *depth, int32_t *token, float *cum_logprob,
                    int32_t *n_nodes, int32_t *frontier_begin,
+                   const float *d_max_seq /* optional [batch]: replaces policy->d_max per sequence */,
                    int32_t *status, void *stream);
+
+/* Adaptive history tracking (Section 3.3 "Adaptive History Tracking"; Section 5.1: window 10, lower
+ * and upper thresholds 2 and 3).  Per sequence b: tau = path_len[b] - 1 (the acceptance length of the
+ * round, from sage_accept) enters a sliding window of the last `window` values
+ * (window_buf[b*window ..], count[b] = values pushed so far; the caller zeroes count once).  When at
+ * least min_samples values are present and their mean is below `lower`, d_max[b] drops by `step`;
+ * above `upper` it rises by `step`; in between it stays (hysteresis); always clamped to [d_lo, d_hi].
+ * The paper fixes the window and the thresholds only; step, clamps and the warm-up rule are this
+ * library's parameters.  d_max[b] can be fed to sage_grow_tree as the sequence's own maximum depth. */
+typedef struct sage_history_policy {
+    int   window;          /* paper: 10 */
+    int   min_samples;     /* 1 .. window: no move before that many values */
+    float lower, upper;    /* paper: 2, 3 */
+    float step;            /* depth change per move */
+    float d_lo, d_hi;      /* clamp range of d_max */
+} sage_history_policy;
+int sage_update_history(const int32_t *path_len, int batch, const sage_history_policy *policy /* host */,
+                        int32_t *window_buf, int32_t *count, float *d_max,
+                        int32_t *status, void *stream);
 
 /* Tree attention mask as per-node ancestor bitsets (Section 2.2: each token attends
  * only to its ancestors; Algorithm 1 TreeAttnMask).  anc[i] has bit j set iff j == i or

@@ -14,7 +14,8 @@ import importlib
 _BINDING_NAMES = (
     "SageError", "SagePolicy", "make_policy", "new_status", "status_string", "lib",
     "sage_expand_topk", "sage_expand_topk_workspace_size", "sage_expand_topk_static", "sage_select_tree",
-    "sage_build_ancestor_mask", "sage_grow_tree", "sage_tree_attention", "sage_tree_attention_workspace_size",
+    "sage_build_ancestor_mask", "sage_grow_tree", "sage_update_history", "make_history_policy",
+    "SageHistoryPolicy", "sage_tree_attention", "sage_tree_attention_workspace_size",
     "sage_accept", "sage_compact_kv",
     "SAGE_OK", "SAGE_ERR_INVALID_ARG", "SAGE_ERR_UNSUPPORTED", "SAGE_ERR_WORKSPACE", "SAGE_ERR_CUDA",
     "SAGE_ERR_TOO_LARGE", "SAGE_STATIC_SCRATCH_BYTES",

@@ -41,6 +41,13 @@ class SagePolicy(ctypes.Structure):
                 ("w_min", ctypes.c_float), ("w_max", ctypes.c_float)]
 
 
+class SageHistoryPolicy(ctypes.Structure):
+    """Mirror of ``sage_history_policy``."""
+    _fields_ = [("window", ctypes.c_int), ("min_samples", ctypes.c_int),
+                ("lower", ctypes.c_float), ("upper", ctypes.c_float), ("step", ctypes.c_float),
+                ("d_lo", ctypes.c_float), ("d_hi", ctypes.c_float)]
+
+
 class SageError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -67,7 +74,9 @@ _lib.sage_select_tree.argtypes = [_vp, _vp, _i, ctypes.POINTER(SagePolicy), _vp,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sage_grow_tree.restype = _i
 _lib.sage_grow_tree.argtypes = [_vp, _vp, _i, _vp, _vp, _i, ctypes.POINTER(SagePolicy), _i,
-                                _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+                                _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sage_update_history.restype = _i
+_lib.sage_update_history.argtypes = [_vp, _i, ctypes.POINTER(SageHistoryPolicy), _vp, _vp, _vp, _vp, _vp]
 _lib.sage_build_ancestor_mask.restype = _i
 _lib.sage_build_ancestor_mask.argtypes = [_vp, _vp, _i, _vp, _vp, _vp]
 _lib.sage_tree_attention.restype = _i
@@ -205,8 +214,8 @@ def sage_select_tree(alpha: torch.Tensor, policy: SagePolicy, *, alpha_row=None,
 
 
 def sage_grow_tree(topk_idx: torch.Tensor, topk_logprob: torch.Tensor, alpha: torch.Tensor, policy: SagePolicy,
-                   tree: Dict[str, torch.Tensor], *, alpha_row=None, n_max: int = SAGE_MAX_NODES, status=None,
-                   stream=None) -> Dict[str, torch.Tensor]:
+                   tree: Dict[str, torch.Tensor], *, alpha_row=None, n_max: int = SAGE_MAX_NODES, d_max_seq=None,
+                   status=None, stream=None) -> Dict[str, torch.Tensor]:
     """One level of dynamic tree construction, in place on ``tree`` (parent, rank, depth, token:
     int32 [batch * SAGE_MAX_NODES]; cum_logprob fp32 of the same length; n_nodes, frontier_begin:
     int32 [batch]).  topk_idx / topk_logprob: [batch * SAGE_MAX_NODES, k]."""
@@ -215,9 +224,25 @@ def sage_grow_tree(topk_idx: torch.Tensor, topk_logprob: torch.Tensor, alpha: to
     code = _lib.sage_grow_tree(_ptr(topk_idx), _ptr(topk_logprob), k, _ptr(alpha), _ptr(alpha_row), batch,
                                ctypes.byref(policy), n_max, _ptr(tree["parent"]), _ptr(tree["rank"]),
                                _ptr(tree["depth"]), _ptr(tree["token"]), _ptr(tree["cum_logprob"]),
-                               _ptr(tree["n_nodes"]), _ptr(tree["frontier_begin"]), _ptr(status), _stream(stream))
+                               _ptr(tree["n_nodes"]), _ptr(tree["frontier_begin"]), _ptr(d_max_seq), _ptr(status),
+                               _stream(stream))
     _check(code, "sage_grow_tree")
     return tree
+
+
+def make_history_policy(window=10, min_samples=None, lower=2.0, upper=3.0, step=1.0, d_lo=3.0, d_hi=8.0):
+    p = SageHistoryPolicy()
+    p.window, p.min_samples = window, window if min_samples is None else min_samples
+    p.lower, p.upper, p.step, p.d_lo, p.d_hi = lower, upper, step, d_lo, d_hi
+    return p
+
+
+def sage_update_history(path_len: torch.Tensor, policy: SageHistoryPolicy, window_buf: torch.Tensor,
+                        count: torch.Tensor, d_max: torch.Tensor, *, status=None, stream=None):
+    """In place: window_buf int32 [batch, window], count int32 [batch], d_max fp32 [batch]."""
+    _check(_lib.sage_update_history(_ptr(path_len), path_len.numel(), ctypes.byref(policy), _ptr(window_buf),
+                                    _ptr(count), _ptr(d_max), _ptr(status), _stream(stream)), "sage_update_history")
+    return d_max
 
 
 def sage_build_ancestor_mask(parent: torch.Tensor, node_offsets: torch.Tensor, *, out=None, status=None, stream=None):

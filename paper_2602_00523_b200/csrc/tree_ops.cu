@@ -290,6 +290,7 @@ struct GrowParams {
     int32_t *parent, *rank, *depth, *token;
     float* cum_logprob;
     int32_t *n_nodes, *frontier_begin;
+    const float* d_max_seq;
     int32_t* status;
 };
 
@@ -306,7 +307,8 @@ __global__ void __launch_bounds__(SAGE_MAX_NODES) grow_tree_kernel(GrowParams p)
     const int level = p.depth[base + fb] + 1;
     const double a = (double)p.alpha[p.alpha_row ? p.alpha_row[b] : b];
     // explicit roundings: no fused multiply-add, so that a host check in plain fp64 sees the same D and W
-    const double D = __dadd_rn((double)p.pol.d_min, __dmul_rn(a, (double)p.pol.d_max - (double)p.pol.d_min));
+    const double d_max = p.d_max_seq ? (double)p.d_max_seq[b] : (double)p.pol.d_max;
+    const double D = __dadd_rn((double)p.pol.d_min, __dmul_rn(a, d_max - (double)p.pol.d_min));
     const double W = __dadd_rn((double)p.pol.w_min, __dmul_rn(1.0 - a, (double)p.pol.w_max - (double)p.pol.w_min));
     if ((double)level > D) {                               // the tree has reached its depth
         if (tid == 0) p.frontier_begin[b] = n;
@@ -353,6 +355,38 @@ __global__ void __launch_bounds__(SAGE_MAX_NODES) grow_tree_kernel(GrowParams p)
         p.n_nodes[b] = min(n + total, p.n_max);
         p.frontier_begin[b] = n;
     }
+}
+
+// ---------------------------------------------------------------------------
+// Adaptive history tracking (Section 3.3; window 10, thresholds 2 and 3 in Section 5.1).
+// One thread per sequence: push tau = path_len - 1 into the sequence's ring of recent
+// acceptance lengths; once `min_samples` values are there, their mean below `lower`
+// lowers the sequence's maximum depth by `step`, above `upper` raises it, clamped to
+// [d_lo, d_hi].  The mean is an exact integer sum divided in fp64.
+// ---------------------------------------------------------------------------
+__global__ void update_history_kernel(const int32_t* __restrict__ path_len, int batch, sage_history_policy pol,
+                                      int32_t* __restrict__ window_buf, int32_t* __restrict__ count,
+                                      float* __restrict__ d_max, int32_t* status) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int pl = path_len[b];
+    const int c = count[b];
+    if (pl < 1 || c < 0) {                          // the root is always accepted: path_len >= 1
+        report_status(status, SAGE_STATUS_BAD_PATH);
+        return;
+    }
+    int32_t* ring = window_buf + (size_t)b * pol.window;
+    ring[c % pol.window] = pl - 1;
+    count[b] = c + 1;
+    const int n = min(c + 1, pol.window);
+    if (n < pol.min_samples) return;
+    long long sum = 0;
+    for (int i = 0; i < n; ++i) sum += ring[i];
+    const double mean = (double)sum / (double)n;
+    float d = d_max[b];
+    if (mean < (double)pol.lower) d = fmaxf(pol.d_lo, d - pol.step);
+    else if (mean > (double)pol.upper) d = fminf(pol.d_hi, d + pol.step);
+    d_max[b] = d;
 }
 
 }  // namespace sage
@@ -421,7 +455,8 @@ extern "C" int sage_compact_kv(void* k_pool, void* v_pool, int64_t layer_stride_
 extern "C" int sage_grow_tree(const int32_t* topk_idx, const float* topk_logprob, int k, const float* alpha,
                               const int32_t* alpha_row, int batch, const sage_tree_policy* policy, int n_max,
                               int32_t* parent, int32_t* rank, int32_t* depth, int32_t* token, float* cum_logprob,
-                              int32_t* n_nodes, int32_t* frontier_begin, int32_t* status, void* stream) {
+                              int32_t* n_nodes, int32_t* frontier_begin, const float* d_max_seq, int32_t* status,
+                              void* stream) {
     if (!topk_idx || !topk_logprob || !alpha || !policy || !parent || !rank || !depth || !token || !cum_logprob ||
         !n_nodes || !frontier_begin)
         return SAGE_ERR_INVALID_ARG;
@@ -432,8 +467,22 @@ extern "C" int sage_grow_tree(const int32_t* topk_idx, const float* topk_logprob
         return SAGE_ERR_INVALID_ARG;
     if (batch == 0) return SAGE_OK;
     GrowParams p{topk_idx, topk_logprob, k, alpha, alpha_row, *policy, n_max, parent, rank, depth, token,
-                 cum_logprob, n_nodes, frontier_begin, status};
+                 cum_logprob, n_nodes, frontier_begin, d_max_seq, status};
     grow_tree_kernel<<<batch, SAGE_MAX_NODES, 0, as_stream(stream)>>>(p);
+    return launch_status();
+}
+
+extern "C" int sage_update_history(const int32_t* path_len, int batch, const sage_history_policy* policy,
+                                   int32_t* window_buf, int32_t* count, float* d_max, int32_t* status,
+                                   void* stream) {
+    if (!path_len || !policy || !window_buf || !count || !d_max || batch < 0) return SAGE_ERR_INVALID_ARG;
+    if (policy->window < 1 || policy->min_samples < 1 || policy->min_samples > policy->window ||
+        !(policy->upper >= policy->lower) || !(policy->d_hi >= policy->d_lo) || !(policy->step >= 0.f))
+        return SAGE_ERR_INVALID_ARG;
+    if (policy->window > 1024) return SAGE_ERR_UNSUPPORTED;
+    if (batch == 0) return SAGE_OK;
+    update_history_kernel<<<(batch + 127) / 128, 128, 0, as_stream(stream)>>>(path_len, batch, *policy, window_buf,
+                                                                              count, d_max, status);
     return launch_status();
 }
 

@@ -80,7 +80,8 @@ def test_grow_tree_argument_validation_needs_no_gpu():
     lib = sage.lib()
     fake = ctypes.c_void_p(0x1000)
     pol = sage.make_policy([])
-    args = [fake, fake, 10, fake, None, 1, ctypes.byref(pol), 64, fake, fake, fake, fake, fake, fake, fake, None, None]
+    args = [fake, fake, 10, fake, None, 1, ctypes.byref(pol), 64, fake, fake, fake, fake, fake, fake, fake, None, None,
+            None]
     bad = list(args); bad[2] = 17
     assert lib.sage_grow_tree(*bad) == sage.SAGE_ERR_UNSUPPORTED
     bad = list(args); bad[7] = 65
@@ -89,3 +90,15 @@ def test_grow_tree_argument_validation_needs_no_gpu():
     assert lib.sage_grow_tree(*bad) == sage.SAGE_ERR_INVALID_ARG
     ok = list(args); ok[5] = 0
     assert lib.sage_grow_tree(*ok) == sage.SAGE_OK
+
+
+def test_update_history_argument_validation_needs_no_gpu():
+    lib = sage.lib()
+    fake = ctypes.c_void_p(0x1000)
+    pol = sage.make_history_policy()
+    assert lib.sage_update_history(fake, 0, ctypes.byref(pol), fake, fake, fake, None, None) == sage.SAGE_OK
+    assert lib.sage_update_history(None, 1, ctypes.byref(pol), fake, fake, fake, None, None) == sage.SAGE_ERR_INVALID_ARG
+    bad = sage.make_history_policy(window=4, min_samples=5)
+    assert lib.sage_update_history(fake, 1, ctypes.byref(bad), fake, fake, fake, None, None) == sage.SAGE_ERR_INVALID_ARG
+    bad = sage.make_history_policy(lower=3.0, upper=2.0)
+    assert lib.sage_update_history(fake, 1, ctypes.byref(bad), fake, fake, fake, None, None) == sage.SAGE_ERR_INVALID_ARG
