@@ -90,7 +90,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.gpu), "-lms", "50"], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except Exception:
             self.proc = None
@@ -257,7 +257,7 @@ def run_cuda(args):
     draft_dev = [t.to(dev) for t in draft_host]
     # target logits need the draft tokens of (round, template): one untimed expansion each
     target_host, target_dev = {}, {}
-    for i in range(total_steps):
+    for i in range(total_steps + 1):                  # one more: the copy pipeline stages one step ahead
         key = (i % ROUNDS, sched[i])
         if key in target_host:
             continue
@@ -295,11 +295,14 @@ def run_cuda(args):
         cur, nxt = tree_buf[i % 2], sel_out[(i + 1) % 2]
         key = (r, sched[i])
         if from_host:
-            draft = draft_in.copy_(draft_host[r], non_blocking=True)
-            target = target_in.copy_(target_host[key], non_blocking=True)
-            q = q_in.copy_(q_host, non_blocking=True)
-            k_pool[:, tree_page, :, :N_NODES, :].copy_(tree_kv_host[0], non_blocking=True)
-            v_pool[:, tree_page, :, :N_NODES, :].copy_(tree_kv_host[1], non_blocking=True)
+            # this step's inputs were copied from pinned host memory on the copy stream while the
+            # previous step computed (two staging slots); the tree's K/V rows go from the staging
+            # slot into their cache page on the device
+            slot = staging[i % 2]
+            torch.cuda.current_stream().wait_event(ev_copied[i % 2])
+            draft, target, q = slot["draft"], slot["target"], slot["q"]
+            k_pool[:, tree_page, :, :N_NODES, :].copy_(slot["tree_kv"][0])
+            v_pool[:, tree_page, :, :N_NODES, :].copy_(slot["tree_kv"][1])
         else:
             draft, target, q = draft_dev[r], target_dev[key], q_dev
         d = sage.sage_expand_topk(draft, K_TOP, K_ENT, parent=cur["next_parent"], rank=cur["next_rank"],
@@ -326,11 +329,27 @@ def run_cuda(args):
             result_dev[MAX_PATH + 1:MAX_PATH + 2].copy_(a["bonus_token"])
             result_dev[MAX_PATH + 2:].copy_(nxt["template_id"])
             result_host.copy_(result_dev, non_blocking=True)
+            ev_consumed[i % 2].record()               # the staging slot may be refilled from here on
         return a, nxt
 
-    draft_in = torch.empty_like(draft_dev[0])
-    target_in = torch.empty_like(draft_dev[0])
-    q_in = torch.empty_like(q_dev)
+    copy_stream = torch.cuda.Stream(device=dev)
+    staging = [{"draft": torch.empty_like(draft_dev[0]), "target": torch.empty_like(draft_dev[0]),
+                "q": torch.empty_like(q_dev), "tree_kv": torch.empty(tree_kv_host.shape, dtype=torch.bfloat16,
+                                                                      device=dev)} for _ in range(2)]
+    ev_copied = [torch.cuda.Event() for _ in range(2)]
+    ev_consumed = [torch.cuda.Event() for _ in range(2)]
+
+    def stage_inputs(i):
+        """Host -> device copies of step i's inputs (draft and target logits, q, the tree's K/V rows),
+        enqueued on the copy stream so that they overlap the previous step's kernels."""
+        slot, r = staging[i % 2], i % ROUNDS
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_consumed[i % 2])        # step i-2 is done with this slot
+            slot["draft"].copy_(draft_host[r], non_blocking=True)
+            slot["target"].copy_(target_host[(r, sched[i])], non_blocking=True)
+            slot["q"].copy_(q_host, non_blocking=True)
+            slot["tree_kv"].copy_(tree_kv_host, non_blocking=True)
+            ev_copied[i % 2].record(copy_stream)
     # tree buffers alternate: sel_out[j] writes into tree_buf[j]'s tensors
     for j in range(2):
         sel_out[j]["template_id"] = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -348,7 +367,11 @@ def run_cuda(args):
             tree_buf[j]["next_parent"].copy_(bank_parent[0])
             tree_buf[j]["next_rank"].copy_(bank_rank[0])
         seen = []
+        if from_host:
+            stage_inputs(0)
         for i in range(args.warmup):
+            if from_host:
+                stage_inputs(i + 1)                   # the next step's copies overlap this step's kernels
             one_round(i, from_host, False)
         barrier()
         sampler = ClockSampler(local)
@@ -358,10 +381,16 @@ def run_cuda(args):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(args.warmup, total_steps):
+            if from_host:
+                # Every timed step issues one full set of host -> device copies (those of the step
+                # after it; the first timed step's own copies ran during the last warm-up step).
+                stage_inputs(i + 1)
             _, nxt = one_round(i, from_host, True)
             if from_host:
                 torch.cuda.current_stream().synchronize()     # the host consumes the result every step
                 seen.append(int(result_host[MAX_PATH + 2]))
+        if from_host:
+            torch.cuda.current_stream().wait_stream(copy_stream)      # the last staged copies end inside the timed region
         e1.record()
         barrier()
         t1 = time.time()
@@ -433,7 +462,9 @@ def run_cuda(args):
             "config": {"workload": WORKLOAD, "parallelism": f"replicas x{world}",
                        "l2": f"inputs larger than L2: {kv_bytes / 1e9:.2f} GB of K/V streamed per step"},
             "e2e": {"value": e2e_value, "unit": "rounds/s", "h2d_bytes_per_step": int(h2d),
-                    "d2h_bytes_per_step": int(result_host.numel() * 4), "ms_per_step": e2e_ms / steps},
+                    "d2h_bytes_per_step": int(result_host.numel() * 4), "ms_per_step": e2e_ms / steps,
+                    "pipeline": "the inputs of step i+1 are copied from pinned host memory on a second stream "
+                                "while step i computes (two staging slots); the host reads every step's result"},
             "gpu_launches": launches * steps,
             "clocks": clocks,
             "roofline": {"kernel": f"tree_attention ({N_LAYERS} stacked layers per launch)", "bound": "tensor",
@@ -461,7 +492,7 @@ def main():
     global N_LAYERS, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=N_LAYERS,
