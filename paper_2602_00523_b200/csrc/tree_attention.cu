@@ -297,6 +297,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_anc[SAGE_MAX_NODES];
+    __shared__ int32_t s_parent[SAGE_MAX_NODES];
     __shared__ int s_flag;
     // 1024-byte alignment: the 128B swizzle pattern repeats every 1024 bytes of address
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -328,17 +329,6 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     if (rpair * kRowsPerCta >= M) return;
     const int n_rtiles = (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1;
 
-    if (tid == 0) s_flag = 0;
-    __syncthreads();
-    if (tid < SAGE_MAX_NODES) {
-        uint64_t a = 0;
-        if (tid < N) {
-            bool bad = false;
-            a = ancestor_bits(p.parent + n0, N, tid, &bad);
-            if (bad) { s_flag = 1; a = 1ull << tid; }
-        }
-        s_anc[tid] = a;
-    }
     // this CTA's slice of the context, in pages
     const int n_pages_seq = (T + kPageSize - 1) / kPageSize;
     const int per_split = (n_pages_seq + p.n_splits - 1) / p.n_splits;
@@ -346,10 +336,26 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     const int pg_end = min(n_pages_seq, pg_begin + per_split);
     const int ns = max(0, pg_end - pg_begin);           // pipeline steps
     const int32_t* pages = p.page_table + (size_t)b * p.max_pages + pg_begin;
-    // page ids of this slice must be valid before the TMA warp uses them as coordinates
+    // One round of global loads: the parent array goes to shared memory (the ancestor walks below
+    // would otherwise be chains of dependent global loads), and the page ids of this slice are
+    // checked before the TMA warp uses them as coordinates.
+    if (tid == 0) s_flag = 0;
+    if (tid < SAGE_MAX_NODES) s_parent[tid] = (tid < N) ? p.parent[n0 + tid] : -1;
+    bool bad_page = false;
     for (int j = tid; j < ns; j += kAttnThreads) {
         const int id = pages[j];
-        if (id < 0 || id >= p.n_pages) s_flag = 2;
+        if (id < 0 || id >= p.n_pages) bad_page = true;
+    }
+    __syncthreads();
+    if (bad_page) s_flag = 2;
+    if (tid < SAGE_MAX_NODES) {
+        uint64_t a = 0;
+        if (tid < N) {
+            bool bad = false;
+            a = ancestor_bits(s_parent, N, tid, &bad);
+            if (bad) { s_flag = 1; a = 1ull << tid; }
+        }
+        s_anc[tid] = a;
     }
     __syncthreads();
     if (s_flag) {
