@@ -819,12 +819,15 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
         !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
         return SAGE_ERR_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SAGE_ERR_CUDA;
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(tree_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
             cudaSuccess)
             return SAGE_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
     dim3 grid(S, row_pairs, n_layers * batch * n_kv_heads);
