@@ -44,11 +44,11 @@ WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefi
 
 
 # DRAM bytes per layer of the attention launch, from the ncu counter capture of the current
-# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 618.83 MB over 9 layers,
+# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 619.08 MB over 9 layers,
 # profiles/tree_attention_kernel_config4_9layers.md).  Traffic grows in proportion to the layer
 # count (every layer streams its own K/V once).  Set to None whenever the kernel changes until the
 # counters are taken again.
-ATTN_DRAM_BYTES_PER_LAYER = 618.83e6 / 9
+ATTN_DRAM_BYTES_PER_LAYER = 619.08e6 / 9
 
 
 def load_peaks():
