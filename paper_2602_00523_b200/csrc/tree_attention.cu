@@ -717,10 +717,11 @@ __global__ void attention_merge_kernel(AttnParams p) {
 
 static int pick_splits(int n_layers, int batch, int n_kv_heads, int G, int max_pages) {
     // One CTA is resident per SM.  Take the smallest slice count whose CTA count fills whole
-    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 8 pages per slice.
+    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 4 pages per slice (short contexts are latency-bound:
+    // more, shorter slices beat fewer CTAs with longer loops; measured at 2k context).
     const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
     const long base = (long)n_layers * batch * n_kv_heads * row_pairs;
-    int s_max = max_pages / 8;
+    int s_max = max_pages / 4;
     if (s_max > 32) s_max = 32;
     if (s_max < 1) s_max = 1;
     int best = 1;
