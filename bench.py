@@ -43,12 +43,10 @@ WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefi
            "page 64 shuffled, 60-node tree, 80 layers, logits 60x152064 fp32"
 
 
-# DRAM bytes per layer of the attention launch, from the ncu counter capture of the current
-# tree_attention_kernel (dram__bytes_read.sum + dram__bytes_write.sum = 619.08 MB over 9 layers,
-# profiles/tree_attention_kernel_config4_9layers.md).  Traffic grows in proportion to the layer
-# count (every layer streams its own K/V once).  Set to None whenever the kernel changes until the
-# counters are taken again.
-ATTN_DRAM_BYTES_PER_LAYER = 619.08e6 / 9
+# DRAM bytes per layer of the attention launch as counted by ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of a 9-layer capture / 9; traffic grows in proportion to the layer count:
+# every layer streams its own K/V once).  None = the kernel changed since the counters were taken.
+ATTN_DRAM_BYTES_PER_LAYER = None
 
 
 def load_peaks():
@@ -79,42 +77,61 @@ def template_schedule(states, steps):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """SM clock, power and clock-event reasons of one GPU while a timed region runs: read-only NVML
+    queries from a thread every ~2 ms (nvidia-smi's loop mode cannot sample a 50 ms region)."""
 
-    def __init__(self, gpu_index):
-        self.rows, self.proc, self.gpu = [], None, gpu_index
+    def __init__(self, uuid=None, index=0):
+        self.rows, self.thread, self.stop_flag, self.h, self.nv = [], None, False, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            if uuid is not None:
+                try:
+                    self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+                except Exception:
+                    self.h = None
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.h = None
+
+    def _loop(self):
+        nv, h = self.nv, self.h
+        while not self.stop_flag:
+            try:
+                self.rows.append((time.time(), float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)),
+                                  int(nv.nvmlDeviceGetCurrentClocksEventReasons(h)),
+                                  nv.nvmlDeviceGetPowerUsage(h) / 1000.0))
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu), "-lms", "50"], stdout=subprocess.PIPE, text=True)
-            threading.Thread(target=self._pump, daemon=True).start()
-        except Exception:
-            self.proc = None
-
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.time(), [v.strip() for v in line.split(",")]))
+        if self.h is None:
+            return
+        self.stop_flag = False
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
 
     def stop(self, t0, t1):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 9] or [r for _, r in self.rows if len(r) >= 9]
+        if self.h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["NVML unavailable"], "samples": 0}
+        self.stop_flag = True
+        self.thread.join()
+        rows = [r for r in self.rows if t0 <= r[0] <= t1] or self.rows
         if not rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        sm = sorted(float(r[1]) for r in rows)
-        reasons = set()
-        for r in rows:
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][2]), "reasons": sorted(reasons),
-                "samples": len(rows), "power_w_max": max(float(r[3]) for r in rows)}
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["no samples"], "samples": 0}
+        nv = self.nv
+        names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
+        reasons = sorted({name for r in rows for bit, name in names.items() if r[2] & bit})
+        sm = sorted(r[1] for r in rows)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": self.sm_max, "reasons": reasons,
+                "samples": len(rows), "power_w_max": max(r[3] for r in rows)}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -176,8 +193,11 @@ def run_reference(args):
     value = 1.0 / full
     sample = "per step: logits side on 6 of 60 rows (x10), attention + compaction of 1 of 8 KV heads of 1 of 80 " \
              "layers (x640); a full round is extrapolated from the sample"
+    # ms_per_step is the measured time of one sampled step (steps x ms_per_step = the timed wall clock);
+    # the round the metric is quoted on is the extrapolation from it, given separately.
     line = {"impl": "reference", "metric": "tree-verify rounds/s", "value": value, "unit": "rounds/s", "n_gpus": 1,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": full * 1e3, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / args.steps * 1e3,
+            "extrapolated_round_ms": full * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": WORKLOAD, "l2": "n/a (CPU)"},
             "cpu_baseline": {"value": value, "unit": "rounds/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -289,6 +309,17 @@ def run_cuda(args):
     result_host = torch.empty(MAX_PATH + 3, dtype=torch.int32).pin_memory()
     result_dev = torch.empty(MAX_PATH + 3, dtype=torch.int32, device=dev)
     attn_events = []
+    other_events = {"expand_draft": [], "expand_target": [], "accept_compact": []}
+
+    def timed_call(name, on, fn):
+        if not on:
+            return fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        r = fn()
+        e1.record()
+        other_events[name].append((e0, e1))
+        return r
 
     def one_round(i, from_host, time_attn):
         r = i % ROUNDS
@@ -305,9 +336,9 @@ def run_cuda(args):
             v_pool[:, tree_page, :, :N_NODES, :].copy_(slot["tree_kv"][1])
         else:
             draft, target, q = draft_dev[r], target_dev[key], q_dev
-        d = sage.sage_expand_topk(draft, K_TOP, K_ENT, parent=cur["next_parent"], rank=cur["next_rank"],
-                                  node_offsets=node_offsets, root_token=root_token, out=out_draft, ws=ws_topk,
-                                  status=status)
+        d = timed_call("expand_draft", time_attn and not from_host, lambda: sage.sage_expand_topk(
+            draft, K_TOP, K_ENT, parent=cur["next_parent"], rank=cur["next_rank"], node_offsets=node_offsets,
+            root_token=root_token, out=out_draft, ws=ws_topk, status=status))
         sage.sage_select_tree(d["alpha"], policy, alpha_row=alpha_row, bank_parent=bank_parent, bank_rank=bank_rank,
                               bank_n_nodes=bank_n, handover=True, out=nxt, status=status)
         if time_attn:
@@ -318,10 +349,15 @@ def run_cuda(args):
         if time_attn:
             e1.record()
             attn_events.append((e0, e1))
-        t = sage.sage_expand_topk(target, 1, 1, out=out_target, ws=ws_topk, status=status)
-        a = sage.sage_accept(cur["next_parent"], d["draft_token"], t["topk_idx"], node_offsets, MAX_PATH,
-                             out=out_accept, status=status)
-        sage.sage_compact_kv(k_pool, v_pool, page_table, seq_len, a["path"], a["path_len"], status=status)
+        t = timed_call("expand_target", time_attn and not from_host, lambda: sage.sage_expand_topk(
+            target, 1, 1, out=out_target, ws=ws_topk, status=status))
+
+        def tail():
+            acc = sage.sage_accept(cur["next_parent"], d["draft_token"], t["topk_idx"], node_offsets, MAX_PATH,
+                                   out=out_accept, status=status)
+            sage.sage_compact_kv(k_pool, v_pool, page_table, seq_len, acc["path"], acc["path_len"], status=status)
+            return acc
+        a = timed_call("accept_compact", time_attn and not from_host, tail)
         seq_len.copy_(seq_len0)                       # the next round starts from the same prefix length
         if from_host:
             result_dev[:MAX_PATH].copy_(a["path"][0])
@@ -363,6 +399,9 @@ def run_cuda(args):
 
     def timed(from_host):
         attn_events.clear()
+        if not from_host:
+            for v in other_events.values():
+                v.clear()
         for j in range(2):                            # both tree buffers restart from template 0
             tree_buf[j]["next_parent"].copy_(bank_parent[0])
             tree_buf[j]["next_rank"].copy_(bank_rank[0])
@@ -374,9 +413,8 @@ def run_cuda(args):
                 stage_inputs(i + 1)                   # the next step's copies overlap this step's kernels
             one_round(i, from_host, False)
         barrier()
-        sampler = ClockSampler(local)
+        sampler = ClockSampler(getattr(torch.cuda.get_device_properties(dev), "uuid", None), local)
         sampler.start()
-        time.sleep(0.25)
         t0 = time.time()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -423,8 +461,70 @@ def run_cuda(args):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)
 
+    def attention_by_tree_size(reps=5):
+        """The 80-layer attention launch alone for trees of 16 ... 60 nodes at the same 16k context
+        (M = nodes x 8 query rows per KV head decides which roof binds: HBM up to about 200 rows, the
+        tensor pipe above).  CUDA events around `reps` launches after two warm-up launches; every launch
+        streams all layers' K/V (far larger than L2)."""
+        from workloads import make_template as mk
+        rows = []
+        for depth, width, n in ((8, 2, 16), (8, 2, 24), (8, 2, 32), (6, 3, 36), (4, 6, 48), (3, 10, 60)):
+            tp = torch.from_numpy(mk(depth, width, n)["parent"]).to(dev)
+            offs = torch.tensor([0, n], dtype=torch.int32, device=dev)
+            qn = q_dev[:, :n].contiguous()
+            on = torch.empty_like(qn)
+            call = lambda: sage.sage_tree_attention(qn, k_pool, v_pool, page_table, seq_len, tp, offs, 1.0 / np.sqrt(D),
+                                                    out=on, ws=ws_attn, status=status)
+            call(); call()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            t_ms = e0.elapsed_time(e1) / reps
+            T = L_PREFIX + n
+            byts = (2.0 * T * HKV * D * 2 + 2.0 * n * HQ * D * 2) * N_LAYERS
+            flop = 4.0 * n * (HQ // HKV) * T * D * HKV * N_LAYERS
+            rows.append({"template": [depth, width, n], "rows_per_kv_head": n * (HQ // HKV), "ms_per_launch": t_ms,
+                         "gbs": byts / (t_ms * 1e-3) / 1e9, "tflops": flop / (t_ms * 1e-3) / 1e12,
+                         "algorithmic_bytes": byts, "flops": flop})
+        return rows
+
+    def attention_latency(passes=2):
+        """Single-layer calls in the latency regime (draft-side attention, level-by-level growth, plain
+        decode): contexts of 2048 and 16384 tokens, trees of 1 / 10 / 60 nodes.  Each pass walks over all
+        layers' K/V, so no call finds its K/V in L2.  Microseconds per call, launch gaps included."""
+        from workloads import chain_tree, make_template as mk
+        rows = []
+        for ctx in (2048, 16384):
+            sl = torch.tensor([ctx], dtype=torch.int32, device=dev)
+            for n, tree in ((1, chain_tree(1)), (10, mk(4, 3, 10)), (60, mk(3, 10, 60))):
+                tp = torch.from_numpy(tree["parent"]).to(dev)
+                offs = torch.tensor([0, n], dtype=torch.int32, device=dev)
+                qs = [q_dev[layer:layer + 1, :n].contiguous() for layer in range(N_LAYERS)]
+                on = torch.empty_like(qs[0])
+
+                def sweep():
+                    for layer in range(N_LAYERS):
+                        sage.sage_tree_attention(qs[layer], k_pool[layer:layer + 1], v_pool[layer:layer + 1], page_table, sl,
+                                                 tp, offs, 1.0 / np.sqrt(D), out=on, ws=ws_attn, status=status)
+                sweep()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(passes):
+                    sweep()
+                e1.record()
+                torch.cuda.synchronize()
+                rows.append({"context": ctx, "nodes": n, "us_per_call": e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)})
+        return rows
+
     ms, attn_ms, clocks, _ = timed(False)
+    other_us = {k: (float(np.mean([a.elapsed_time(b) for a, b in v])) * 1e3 if v else None) for k, v in other_events.items()}
     layer_us = None if args.no_per_layer else per_layer_attention_us()
+    by_tree = None if args.no_sweeps else attention_by_tree_size()
+    latency = None if args.no_sweeps else attention_latency()
     if int(status.item()) != 0:
         raise RuntimeError("device status: " + sage.status_string(int(status.item())))
     e2e_ms, _, _, seen = timed(True)
@@ -453,8 +553,25 @@ def run_cuda(args):
                             "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
                                       f"rows), attention, acceptance and compaction of 1 of the {N_LAYERS} layers; "
                                       "the other layers are extrapolated"}
-        n_splits_gt1 = sage.sage_tree_attention_workspace_size(N_LAYERS, 1, N_NODES, HQ, HKV, D, used_pages) > 16
-        launches = 3 + 2 + (2 if n_splits_gt1 else 1) + 2 + 1 + 2
+        launches = 3 + 2 + 2 + 2 + 1 + 2      # expand (3), select + hand-over, attention + merge, target top-1 (2), accept, compact (2)
+        # Which tensor peak applies: the burst figure when the SM clock stayed at its maximum through the
+        # timed region, the sustained one when the power cap pulled it down.  Both fractions are printed.
+        sm, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+        burst = bool(sm and sm_max and sm >= 0.97 * sm_max and "sw_power_cap" not in clocks.get("reasons", []))
+        peak_tf = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+        hbm_entry = None
+        if by_tree is not None:
+            for row in by_tree:
+                row["frac_hbm"] = row["gbs"] / peaks["hbm_gbs"]
+                row["frac_bf16_burst"] = row["tflops"] / peaks["bf16_tflops"]
+                row["bound"] = "hbm" if row["rows_per_kv_head"] * 1.0 < peaks["bf16_tflops"] * 1e3 / peaks["hbm_gbs"] else "tensor"
+            r24 = by_tree[1]
+            hbm_entry = {"kernel": f"tree_attention, 24-node (8,2) tree, {N_LAYERS} stacked layers, 16k context",
+                         "bound": "hbm", "achieved": r24["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": r24["frac_hbm"], "traffic": None, "ms_per_launch": r24["ms_per_launch"],
+                         "algorithmic_bytes": r24["algorithmic_bytes"], "target_frac": 0.70,
+                         "target_met": bool(r24["frac_hbm"] >= 0.70), "peak_source": peaks["source"] + " (copy bandwidth)"}
+        logits_bytes = float(N_NODES) * V * 4
         line = {
             "metric": "tree-verify rounds/s", "value": value, "unit": "rounds/s", "n_gpus": world, "steps": steps,
             "warmup": args.warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
@@ -467,19 +584,40 @@ def run_cuda(args):
                                 "while step i computes (two staging slots); the host reads every step's result"},
             "gpu_launches": launches * steps,
             "clocks": clocks,
-            "roofline": {"kernel": f"tree_attention ({N_LAYERS} stacked layers per launch)", "bound": "tensor",
-                         "achieved": ach_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": ach_tf / peaks["bf16_tflops_sustained"],
+            "roofline": {"kernel": f"tree_attention, 60-node tree ({N_LAYERS} stacked layers per launch)", "bound": "tensor",
+                         "achieved": ach_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": ach_tf / peak_tf,
+                         "frac_of_burst_peak": ach_tf / peaks["bf16_tflops"],
+                         "frac_of_sustained_peak": ach_tf / peaks["bf16_tflops_sustained"],
+                         "peak_regime": "burst (SM clock at maximum during the timed region)" if burst else
+                                        "sustained (SM clock below maximum / power cap active during the timed region)",
+                         "ms_x_sm_mhz": None if not sm else attn_ms * sm,
                          "traffic": None if ATTN_DRAM_BYTES_PER_LAYER is None else ATTN_DRAM_BYTES_PER_LAYER * N_LAYERS,
                          "traffic_unit": "bytes per launch (ncu DRAM read+write on a 9-layer capture, scaled by layers)",
                          "algorithmic_bytes": kv_bytes,
-                         "peak_source": peaks["source"] + " (sustained bf16)", "ms_per_launch": attn_ms,
+                         "peak_source": peaks["source"], "ms_per_launch": attn_ms,
                          "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                 "frac": ach_gb / peaks["hbm_gbs"]}},
+                                 "frac": ach_gb / peaks["hbm_gbs"],
+                                 "note": "480 query rows per KV head: above the ridge, the tensor roof binds; the "
+                                         "70 % HBM target applies to the HBM-bound trees (roofline_hbm_bound)"}},
+            "roofline_hbm_bound": hbm_entry,
+            "attention_by_tree_size": by_tree,
+            "attention_latency": latency,
+            "other_launches": {
+                "expand_topk_draft_k10": None if not other_us["expand_draft"] else {
+                    "us": other_us["expand_draft"], "gbs": logits_bytes / (other_us["expand_draft"] * 1e-6) / 1e9,
+                    "frac_hbm": logits_bytes / (other_us["expand_draft"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                    "algorithmic_bytes": logits_bytes, "launches": 3},
+                "expand_topk_target_k1": None if not other_us["expand_target"] else {
+                    "us": other_us["expand_target"], "gbs": logits_bytes / (other_us["expand_target"] * 1e-6) / 1e9,
+                    "frac_hbm": logits_bytes / (other_us["expand_target"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                    "algorithmic_bytes": logits_bytes, "launches": 2},
+                "accept_compact": None if not other_us["accept_compact"] else {
+                    "us": other_us["accept_compact"], "launches": 3,
+                    "note": f"{N_LAYERS} layers; at most 9 rows x 8 heads x 256 B x 2 pools moved per layer: latency-bound"}},
             "attention_per_layer": None if layer_us is None else {
                 "us_per_call": layer_us, "tflops": flops / N_LAYERS / (layer_us * 1e-6) / 1e12,
                 "gbs": kv_bytes / N_LAYERS / (layer_us * 1e-6) / 1e9,
-                "note": "80 single-layer calls walking over all layers' K/V (split-K + merge kernels, launch "
+                "note": "80 single-layer calls walking over all layers' K/V (attention + merge kernels, launch "
                         "gaps included)"},
             "cpu_baseline": cpu_baseline,
         }
@@ -499,6 +637,8 @@ def main():
                     help="stacked layers per round (the workload has 80; fewer only for small profiler captures)")
     ap.add_argument("--no-per-layer", action="store_true",
                     help="skip the layer-by-layer attention timing (profiler launch lists of the round alone)")
+    ap.add_argument("--no-sweeps", action="store_true",
+                    help="skip the tree-size sweep and the latency sweep of the attention call")
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip timing the CPU oracle (profiler captures)")
     args = ap.parse_args()

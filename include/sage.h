@@ -206,7 +206,10 @@ int sage_build_ancestor_mask(const int32_t *parent, const int32_t *node_offsets,
  * q, out: bf16 [n_layers][sum_nodes][n_q_heads][head_dim]; `sum_nodes` is the node
  * capacity of those buffers (>= node_offsets[batch]).  Softmax and accumulation in
  * fp32.  Rows of the cache beyond L_b+N_b may hold anything (NaN included).
- * ws: sage_tree_attention_workspace_size(...) bytes. */
+ * ws: sage_tree_attention_workspace_size(...) bytes (a fixed amount per streaming multiprocessor of
+ * the current device, independent of the problem size: the kernel is one resident thread block
+ * per multiprocessor, and each keeps at most two partial results for sequences that a work
+ * boundary cuts). */
 int sage_tree_attention(const void *q, const void *k_pool, const void *v_pool,
                         int64_t layer_stride_elems, int n_layers, int n_pages,
                         const int32_t *page_table, int max_pages_per_seq, const int32_t *seq_len,
@@ -231,13 +234,26 @@ int sage_accept(const int32_t *parent, const int32_t *draft_token, const int32_t
 /* KV-cache update with the accepted tokens (Algorithm 1; Section 3.3 "Phase 2").  In place,
  * for every layer, KV head and j < path_len[b]: the K and V rows at logical position
  * L_b + path[b][j] move to L_b + j (all rows are read before any is written), then
- * seq_len[b] += path_len[b].  No other byte of the pools changes. */
+ * seq_len[b] += path_len[b].  No other byte of the pools changes.  A sequence whose path is not a
+ * root path (entries not strictly increasing from 0, or path_len outside [0, max_path]) or whose
+ * pages are out of range is reported in `status` and left untouched: no row moves and its
+ * seq_len does not advance. */
 int sage_compact_kv(void *k_pool, void *v_pool, int64_t layer_stride_elems, int n_layers, int n_pages,
                     const int32_t *page_table, int max_pages_per_seq, int32_t *seq_len,
                     const int32_t *path, const int32_t *path_len, int batch, int max_path,
                     int n_kv_heads, int head_dim, int page_size, int32_t *status, void *stream);
 
 const char *sage_status_string(int code);
+
+/* Diagnostics for the failure path of sage_tree_attention (no counterpart in the paper).  Every
+ * on-device wait of that kernel has a cycle budget; when one runs out the thread block records
+ * SAGE_STATUS_TIMEOUT, waits (again bounded) for its own copies and tensor-core work in flight,
+ * releases its tensor memory and returns, so the context stays usable.  This call sets, for all
+ * later sage_tree_attention calls of the process, the budget in clock cycles (<= 0 restores the
+ * default of about two seconds) and, when producer_off != 0, keeps the copy warp from issuing
+ * anything, so that the first consumer wait is one that nothing will ever satisfy.  Tests use it
+ * to run the time-out path without faulting or hanging the device; leave it alone otherwise. */
+void sage_debug_attention_waits(long long wait_cycles, int producer_off);
 
 #ifdef __cplusplus
 }

@@ -88,6 +88,8 @@ _lib.sage_accept.restype = _i
 _lib.sage_accept.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.sage_compact_kv.restype = _i
 _lib.sage_compact_kv.argtypes = [_vp, _vp, _i64, _i, _i, _vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.sage_debug_attention_waits.restype = None
+_lib.sage_debug_attention_waits.argtypes = [ctypes.c_longlong, _i]
 _lib.sage_status_string.restype = ctypes.c_char_p
 _lib.sage_status_string.argtypes = [_i]
 
@@ -281,6 +283,12 @@ def sage_tree_attention(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Ten
                                     ws.numel(), _ptr(status), _stream(stream))
     _check(code, "sage_tree_attention")
     return out
+
+
+def sage_debug_attention_waits(wait_cycles: int = 0, producer_off: bool = False) -> None:
+    """Cycle budget of the attention kernel's on-device waits (0 = default) and, for tests of the
+    time-out path, a switch that keeps its copy warp from issuing anything."""
+    _lib.sage_debug_attention_waits(int(wait_cycles), 1 if producer_off else 0)
 
 
 def sage_accept(parent, draft_token, target_argmax, node_offsets, max_path: int, *, out=None, status=None, stream=None):

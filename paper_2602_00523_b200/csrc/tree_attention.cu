@@ -1,23 +1,34 @@
 // Tree-masked verification attention over a paged bf16 KV cache (Section 2.2;
 // Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2), sm_100a.
 //
-// Flash-decoding layout.  The N tree nodes x G query heads that share one KV head
-// form M = N*G query rows (<= 512).  A CTA owns up to two 128-row tiles of them and
-// one slice of the context (split-K).  The pipeline step is one 64-token page:
-//   TMA      : K and V pages -> 128B-swizzled shared memory, two 5-page rings, mbarriers
-//   tcgen05  : S_t = Q_t K^T (128 x 64, fp32) into TMEM; one warp per row tile issues, through
+// Work decomposition.  The N tree nodes x G query heads that share one KV head form
+// M = N*G query rows (<= 512).  An *item* is one (layer, sequence, KV head); its work
+// is measured in steps of 128 keys (two 64-token pages).  All items are laid end to
+// end and cut into equal ranges of steps, one range per *gang*; a gang is the 1 or 2
+// CTAs (one per 256 query rows) that walk the same range side by side, so that the
+// second CTA finds the K/V of the first in L2.  A kernel launch is one resident CTA
+// per SM that loops over the segments of its range: whole items write their output
+// directly, items cut by a range boundary leave unnormalised partial results that
+// attention_merge_kernel combines.  Nothing waits on another CTA.
+//
+// Inside a CTA (384 threads), per 128-key step and 128-row tile t:
+//   TMA      : K and V tiles (2 pages x 2 d-halves) -> 128B-swizzled shared memory, rings of
+//              3 K tiles and 2 V tiles, mbarriers; the two query tiles also arrive by TMA
+//   tcgen05  : S_t = Q_t K^T (128 x 128, fp32) into TMEM; one warp issues for both row tiles, through
 //              one elected lane, with warp-uniform descriptor arithmetic
-//   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S, online
-//              softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back into TMEM
+//   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S in four 32-column
+//              chunks, online softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back
+//              into TMEM over the first 64 columns of S_t
 //   tcgen05  : O_t += P_t V with P as the TMEM A operand, V MN-major from shared memory
-// Every row tile has two S buffers (even / odd pages), so the tensor pipe computes the
-// scores of page j+1 while the warpgroup is busy with page j and never waits for it.
-// TMEM map (512 columns): tile t owns S_t,even [128t, 128t+64), S_t,odd [128t+64, 128t+128)
-// (P overlays the first 32 columns of its S buffer) and O_t [256+128t, 384+128t).
-// Slices are merged by attention_merge_kernel (warp per output row).  All waits are
-// bounded: on expiry the CTA records SAGE_STATUS_TIMEOUT, drains its copies, frees its
-// TMEM and returns.
+// A 128 x 64 score MMA occupies the tensor pipe exactly as long as a 128 x 128 one (64 clocks
+// per K=16 slice, measured), hence the 128-key step.  The two row tiles alternate on the
+// tensor pipe: while one tile's warpgroup runs its softmax, the pipe works on the other tile.
+// TMEM map (512 columns): S_t [128t, 128t+128), O_t [256+128t, 384+128t).
+// All waits are bounded: on expiry the CTA records SAGE_STATUS_TIMEOUT, waits (bounded) for
+// its copies and MMAs in flight, frees its TMEM and returns.
 #include <cuda.h>
+
+#include <mutex>
 
 #include "sage_common.cuh"
 
@@ -25,42 +36,52 @@ namespace sage {
 
 constexpr int kRowTile = 128;                  // query rows per MMA tile
 constexpr int kRowsPerCta = 2 * kRowTile;
-constexpr int kStages = 5;                     // depth of the K ring and of the V ring, in pages
-constexpr int kPageBytes = kPageSize * kHeadDim * 2;        // one (page, head) tile: 16 KB
-constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // one 64-wide d-half of a page: 8 KB
+constexpr int kStepKeys = 2 * kPageSize;       // keys per pipeline step
+constexpr int kKStages = 3;                    // K tiles in flight
+constexpr int kVStages = 2;                    // V tiles in flight
+constexpr int kRing = 4;                       // barrier pairs of the copy ring (ring steps in flight <= 2)
+constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // one TMA box: 64 keys x 64-wide d-half = 8 KB
+constexpr int kTileHalfBytes = kStepKeys * 64 * 2;          // one d-half of a 128-key tile: 16 KB
+constexpr int kTileBytes = 2 * kTileHalfBytes;              // K or V tile of one step: 32 KB
 constexpr int kQTileBytes = kRowTile * kHeadDim * 2;        // 32 KB
 constexpr int kQHalfBytes = kRowTile * 64 * 2;              // one 64-wide d-half of a Q tile: 16 KB
-constexpr int kAttnThreads = 352;              // 2 softmax warpgroups + TMA warp + one MMA warp per row tile
-constexpr int kSmemBytes = 2 * kQTileBytes + 2 * kStages * kPageBytes + 1024 /*align*/ + 512 /*barriers*/;
-constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: far beyond any legitimate wait
+constexpr int kAttnThreads = 384;              // 2 softmax warpgroups + one warpgroup of TMA warp, MMA warp and two idle warps
+constexpr int kMinSteps = 2;                   // no range shorter than this (short contexts are latency-bound)
+constexpr long long kWaitCyclesDefault = 4000000000ll;   // ~2 s at 2 GHz: far beyond any legitimate wait
 
 struct AttnParams {
-    const __nv_bfloat16* q;
     __nv_bfloat16* out;
-    float* part_o;     // [layer][split][sum_nodes*Hq][128]   unnormalised
-    float* part_ml;    // [layer][split][sum_nodes*Hq][2]     (reference max in log2 units, l)
+    float* part_o;     // [gang][2][gang member][256 rows][128]   unnormalised
+    float* part_ml;    // [gang][2][gang member][256 rows][2]     (reference max in log2 units, l)
     const int32_t* page_table;
     const int32_t* seq_len;
     const int32_t* parent;
     const int32_t* node_offsets;
     int32_t* status;
     int n_layers, batch, sum_nodes, n_pages, max_pages;
-    int Hq, Hkv, G, n_splits;
-    float scale_log2;  // sm_scale * log2(e)
+    int Hq, Hkv, G;
+    int n_gangs, n_rp;         // gangs in the launch, CTAs per gang (row pairs of the largest possible tree)
+    float scale_log2;          // sm_scale * log2(e)
+    long long wait_cycles;     // budget of every on-device wait
+    int producer_off;          // diagnostics: the TMA warp issues no copies (every consumer wait then runs out)
 };
 
-struct __align__(8) Barriers {
-    uint64_t k_full[kStages], k_empty[kStages];
-    uint64_t v_full[kStages], v_empty[kStages];
-    uint64_t s_full[2][2];     // [row tile][page parity]: scores of a page are in TMEM
-    uint64_t p_full[2][2];     // [row tile][page parity]: probabilities of a page are in TMEM
-    uint64_t pv_done[2];       // [row tile]: completes once per page, when its P V product has finished
-    uint64_t o_full[2];        // [row tile]: every MMA of the tile has finished
-    uint64_t q_ready;          // the query tiles are staged in shared memory
+struct __align__(16) Shared {
+    uint64_t kv_full[kRing];   // ring step r: the K tile of its step and the V tile of the step before have landed
+    uint64_t kv_done[kRing];   // ring step r: every MMA that reads those tiles has finished
+    uint64_t s_full[2];        // [row tile]: scores of a step are in TMEM
+    uint64_t p_full[2];        // [row tile]: probabilities of a step are in TMEM
+    uint64_t o_full[2];        // [row tile]: every MMA of the segment has finished
+    uint64_t q_free;           // the segment's last score MMAs have read the query tiles
+    uint64_t q_ready;          // the query tiles of the segment are in shared memory
+    uint64_t drain;            // abort path: everything issued so far has retired
+    long long range_begin, range_end;
+    int first_lg, first_b, first_s0;
     uint32_t tmem_base;
     volatile int abort;
 };
-static_assert(sizeof(Barriers) <= 512, "barrier block outgrew its shared-memory reservation");
+constexpr int kSmemBytes = 1024 /*align*/ + 2 * kQTileBytes + (kKStages + kVStages) * kTileBytes + (int)sizeof(Shared);
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -81,19 +102,24 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* bars, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, const AttnParams& p) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
-        if (bars->abort) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            bars->abort = 1;
-            report_status(status, SAGE_STATUS_TIMEOUT);
+        if (sh->abort) return false;
+        if (clock64() - t0 > p.wait_cycles) {
+            sh->abort = 1;
+            report_status(p.status, SAGE_STATUS_TIMEOUT);
             return false;
         }
     }
+}
+// Used on the abort path only: gives up silently after the budget.
+__device__ __forceinline__ void mbar_wait_quiet(uint64_t* bar, uint32_t parity, long long budget) {
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity) && clock64() - t0 < budget) {}
 }
 
 // ---- TMA ----------------------------------------------------------------------
@@ -102,6 +128,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar)) : "memory");
 }
 
 // ---- tcgen05 --------------------------------------------------------------------
@@ -119,20 +151,22 @@ __device__ __forceinline__ void tc_commit(bool leader, uint64_t* bar) {
     if (leader)
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Shared-memory matrix descriptors are passed as (low word, high word): only the low word (start
+// address and leading byte offset) varies between the MMAs of a kernel, so the issuing thread keeps
+// 32-bit values and the 64-bit operand is assembled next to the instruction.
 // D[tmem] (+)= A[smem desc] * B[smem desc]
-template <bool kAcc>
-__device__ __forceinline__ void mma_ss(bool leader, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
-    if (leader)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(kAcc ? 1 : 0) : "memory");
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(bool leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    if (leader)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (quadrant*32 + i)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -145,7 +179,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
         "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
@@ -174,16 +208,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
-// offsets in 16-byte units, version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+// offsets in 16-byte units, version 1, 128-byte swizzle.  Low word: address and leading offset;
+// high word: stride offset (1024 bytes between 8-row groups everywhere here), version, swizzle.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
 }
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N as given.
 constexpr uint32_t idesc_f16(uint32_t n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
-constexpr uint32_t kIdescQK = idesc_f16(kPageSize);              // S (128 x 64): A, B both K-major
+constexpr uint32_t kIdescQK = idesc_f16(kStepKeys);              // S (128 x 128): A, B both K-major
 constexpr uint32_t kIdescPV = idesc_f16(kHeadDim) | (1u << 16);  // O (128 x 128): B (= V) MN-major
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -235,44 +270,78 @@ __device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float& p0, float& p1)
     p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
 }
 
-// One 64-key half of a softmax step for one query row: p = 2^(s * scale + neg_ref), packed to
-// bf16 pairs (in place, over the first 32 words of `sr`), and their fp32 sum.  kEmu of every 8
-// column pairs take the FMA-pipe exp2.  Written in stages over the whole row so that neighbouring
-// instructions are independent: a softmax warp mostly runs alone on its scheduler.
+#ifndef SAGE_EXP2_FMA_PAIRS
+#define SAGE_EXP2_FMA_PAIRS 1       // of every 8 column pairs, evaluated on the FMA pipe instead of the SFU
+#endif
+
+// Maximum of 32 raw scores of one query row, folded into mx.
+__device__ __forceinline__ void max_chunk(const uint32_t* sr, float& mx) {
+    float m4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float mq = max3(__uint_as_float(sr[q * 8]), __uint_as_float(sr[q * 8 + 1]), __uint_as_float(sr[q * 8 + 2]));
+        mq = max3(mq, __uint_as_float(sr[q * 8 + 3]), __uint_as_float(sr[q * 8 + 4]));
+        mq = max3(mq, __uint_as_float(sr[q * 8 + 5]), __uint_as_float(sr[q * 8 + 6]));
+        m4[q] = fmaxf(mq, __uint_as_float(sr[q * 8 + 7]));
+    }
+    mx = fmaxf(max3(mx, m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+}
+
+// 32 score columns of one query row: p = 2^(s * scale + neg_ref) packed to 16 bf16 pairs, and the
+// fp32 sums of p in `acc`.  kEmu of every 8 column pairs take the FMA-pipe exp2.  Written in stages
+// over the chunk so that neighbouring instructions are independent.
 template <int kEmu>
-__device__ __forceinline__ float softmax_half(uint32_t (&sr)[64], float scale, float neg_ref) {
+__device__ __forceinline__ void exp_chunk(const uint32_t* sr, float scale, float neg_ref, uint32_t* pk,
+                                          uint64_t (&acc)[2]) {
     const uint64_t scale2 = f2_pack(scale, scale), nref2 = f2_pack(neg_ref, neg_ref);
-    uint64_t x2[32];
 #pragma unroll
-    for (int i = 0; i < 32; ++i)
-        x2[i] = f2_fma(f2_pack(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), scale2, nref2);
+    for (int h = 0; h < 2; ++h) {
+        uint64_t x2[8];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        float p0, p1;
-        if ((i & 7) < kEmu) {
-            exp2_pair_fma(x2[i], p0, p1);
-        } else {
-            float x0, x1;
-            f2_unpack(x2[i], x0, x1);
-            p0 = fast_exp2(x0);
-            p1 = fast_exp2(x1);
+        for (int i = 0; i < 8; ++i)
+            x2[i] = f2_fma(f2_pack(__uint_as_float(sr[16 * h + 2 * i]), __uint_as_float(sr[16 * h + 2 * i + 1])), scale2, nref2);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float p0, p1;
+            if (i < kEmu) {
+                exp2_pair_fma(x2[i], p0, p1);
+            } else {
+                float x0, x1;
+                f2_unpack(x2[i], x0, x1);
+                p0 = fast_exp2(x0);
+                p1 = fast_exp2(x1);
+            }
+            x2[i] = f2_pack(p0, p1);
         }
-        x2[i] = f2_pack(p0, p1);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i & 1] = f2_add(acc[i & 1], x2[i]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float p0, p1;
+            f2_unpack(x2[i], p0, p1);
+            pk[8 * h + i] = pack_bf16(p0, p1);
+        }
     }
-    uint64_t acc[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] = x2[i];
-#pragma unroll
-    for (int i = 4; i < 32; ++i) acc[i & 3] = f2_add(acc[i & 3], x2[i]);
+}
+
+// Scores of keys this row may not see become -inf: tree slot jt is visible iff it is an
+// ancestor of (or is) the row's node; positions past the tree are never visible.
+__device__ __forceinline__ void mask_chunk(uint32_t* sr, int pos0, int L, int N, uint64_t anc) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        float p0, p1;
-        f2_unpack(x2[i], p0, p1);
-        sr[i] = pack_bf16(p0, p1);
+        const int jt = pos0 + i - L;                      // tree slot; < 0 = prefix
+        const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
+        if (!vis) sr[i] = 0xff800000u;                    // -inf
     }
-    float a, b;
-    f2_unpack(f2_add(f2_add(acc[0], acc[1]), f2_add(acc[2], acc[3])), a, b);
-    return a + b;
+}
+
+// The 128 scores of a step for one query row, TMEM -> registers: four loads, one wait.
+__device__ __forceinline__ void load_scores(uint32_t s_taddr, uint32_t (&sr)[128]) {
+    tmem_ld32(s_taddr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+    tmem_ld32(s_taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+    tmem_ld32(s_taddr + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+    tmem_ld32(s_taddr + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+    tmem_wait_ld();
 }
 
 // O row *= alpha for the 32 rows of this warp (rare: only when a row maximum grew by more than 2^8).
@@ -289,383 +358,499 @@ __device__ __noinline__ void rescale_o_rows(uint32_t o_taddr, float alpha) {
     tmem_wait_st();
 }
 
-#ifndef SAGE_EXP2_FMA_PAIRS
-#define SAGE_EXP2_FMA_PAIRS 1       // of every 8 column pairs (measured best with both warpgroups busy at once)
-#endif
+// ---- schedule: items, ranges, segments ---------------------------------------------------
+struct Item { int n0, N, L, steps, rp; };     // steps == 0: the sequence is skipped (and reported)
+
+__device__ __forceinline__ Item load_item(const AttnParams& p, int b, int* err) {
+    Item it;
+    it.n0 = p.node_offsets[b];
+    it.N = p.node_offsets[b + 1] - it.n0;
+    it.L = p.seq_len[b];
+    it.steps = 0;
+    it.rp = 0;
+    if (it.N < 1 || it.N > SAGE_MAX_NODES || it.n0 < 0 || it.n0 + it.N > p.sum_nodes) {
+        *err = SAGE_STATUS_BAD_TREE;
+        return it;
+    }
+    if (it.L < 0 || (long long)it.L + it.N > (long long)p.max_pages * kPageSize) {
+        *err = SAGE_STATUS_BAD_PAGE;
+        return it;
+    }
+    it.steps = (it.L + it.N + kStepKeys - 1) / kStepKeys;
+    it.rp = (it.N * p.G + kRowsPerCta - 1) / kRowsPerCta;
+    return it;
+}
+
+// Steps of all sequences of one (layer, KV head); called by a whole warp.
+__device__ __forceinline__ int steps_per_head(const AttnParams& p, int lane, int* err) {
+    int total = 0;
+    for (int b0 = 0; b0 < p.batch; b0 += 32) {
+        int s = 0;
+        if (b0 + lane < p.batch) s = load_item(p, b0 + lane, err).steps;
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        total += s;
+    }
+    return total;
+}
+__device__ __forceinline__ int active_gangs(long long W, int n_gangs) {
+    long long a = W / kMinSteps;
+    if (a < 1) a = 1;
+    return a < n_gangs ? (int)a : n_gangs;
+}
+__device__ __forceinline__ long long gang_begin(long long W, int n_act, int gang) { return (long long)gang * W / n_act; }
+// Gang whose range holds position pos: the largest k with gang_begin(k) <= pos.
+__device__ __forceinline__ int gang_of(long long W, int n_act, long long pos) {
+    return (int)(((pos + 1) * n_act - 1) / W);
+}
+// Sequence b and step s0 inside it for offset `off` into one (layer, KV head); whole warp.
+__device__ __forceinline__ void locate(const AttnParams& p, int lane, int off, int* b_out, int* s0_out) {
+    int run = 0, err = 0;
+    *b_out = p.batch;
+    *s0_out = 0;
+    for (int b0 = 0; b0 < p.batch; b0 += 32) {
+        int s = 0;
+        if (b0 + lane < p.batch) s = load_item(p, b0 + lane, &err).steps;
+        int inc = s;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, run + inc > off);
+        if (hit) {
+            const int l = __ffs(hit) - 1;
+            const int incl = __shfl_sync(0xffffffffu, inc, l), sl = __shfl_sync(0xffffffffu, s, l);
+            *b_out = b0 + l;
+            *s0_out = off - (run + incl - sl);
+            return;
+        }
+        run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+}
+
+struct Seg { int layer, g, b, n0, N, L, s0, s1, steps, rp; bool at_range_begin; };
+
+// Walks the segments of a range; every thread that needs them runs its own copy.
+struct SegIter {
+    int remaining;      // steps of the range still to hand out
+    int lg, b, s0;
+    bool fresh;         // nothing handed out yet
+    __device__ __forceinline__ void init(const Shared* sh) {
+        remaining = (int)(sh->range_end - sh->range_begin);
+        lg = sh->first_lg;
+        b = sh->first_b;
+        s0 = sh->first_s0;
+        fresh = true;
+    }
+    __device__ __forceinline__ bool next(const AttnParams& p, Seg& sg) {
+        int skipped = 0;
+        while (remaining > 0 && b < p.batch && skipped <= p.batch) {
+            int err = 0;
+            const Item it = load_item(p, b, &err);
+            if (it.steps == 0) {
+                ++skipped;
+                if (++b == p.batch) { b = 0; ++lg; }
+                continue;
+            }
+            const int s1 = (it.steps - s0 <= remaining) ? it.steps : s0 + remaining;
+            sg.layer = lg / p.Hkv; sg.g = lg % p.Hkv; sg.b = b;
+            sg.n0 = it.n0; sg.N = it.N; sg.L = it.L;
+            sg.s0 = s0; sg.s1 = s1; sg.steps = it.steps; sg.rp = it.rp;
+            sg.at_range_begin = fresh;
+            fresh = false;
+            remaining -= s1 - s0;
+            if (s1 == it.steps) {
+                s0 = 0;
+                if (++b == p.batch) { b = 0; ++lg; }
+            } else {
+                s0 = s1;
+            }
+            return true;
+        }
+        return false;
+    }
+};
 
 __global__ void __launch_bounds__(kAttnThreads, 1)
-tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
+tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qmap,
+                      const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_anc[SAGE_MAX_NODES];
-    __shared__ int32_t s_parent[SAGE_MAX_NODES];
-    __shared__ int s_flag;
     // 1024-byte alignment: the 128B swizzle pattern repeats every 1024 bytes of address
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                 // [2 tiles][2 d-halves][128 rows][128 B]
-    uint8_t* sK = smem + 2 * kQTileBytes;               // [kStages][2 d-halves][64 keys][128 B]
-    uint8_t* sV = sK + kStages * kPageBytes;            // [kStages][2 d-halves][64 keys][128 B]
-    Barriers* bars = reinterpret_cast<Barriers*>(sV + kStages * kPageBytes);
+    uint8_t* sK = sQ + 2 * kQTileBytes;                 // [kKStages][2 d-halves][128 keys][128 B]
+    uint8_t* sV = sK + kKStages * kTileBytes;           // [kVStages][2 d-halves][128 keys][128 B]
+    Shared* sh = reinterpret_cast<Shared*>(sV + kVStages * kTileBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int split = blockIdx.x, rpair = blockIdx.y;
-    const int g = blockIdx.z % p.Hkv;
-    const int b = (blockIdx.z / p.Hkv) % p.batch;
-    const int layer = blockIdx.z / (p.Hkv * p.batch);
+    const int member = blockIdx.x % p.n_rp, gang = blockIdx.x / p.n_rp;
 
-    // ---- uniform early exits (before any barrier or TMEM is touched)
-    const int n0 = p.node_offsets[b];
-    const int N = p.node_offsets[b + 1] - n0;
-    const int L = p.seq_len[b];
-    if (N < 1 || N > SAGE_MAX_NODES || n0 < 0 || n0 + N > p.sum_nodes) {
-        if (tid == 0) report_status(p.status, SAGE_STATUS_BAD_TREE);
-        return;
-    }
-    const int T = L + N;
-    if (L < 0 || T > p.max_pages * kPageSize) {
-        if (tid == 0) report_status(p.status, SAGE_STATUS_BAD_PAGE);
-        return;
-    }
-    const int M = N * p.G;
-    if (rpair * kRowsPerCta >= M) return;
-    const int n_rtiles = (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1;
-
-    // this CTA's slice of the context, in pages
-    const int n_pages_seq = (T + kPageSize - 1) / kPageSize;
-    const int per_split = (n_pages_seq + p.n_splits - 1) / p.n_splits;
-    const int pg_begin = split * per_split;
-    const int pg_end = min(n_pages_seq, pg_begin + per_split);
-    const int ns = max(0, pg_end - pg_begin);           // pipeline steps
-    const int32_t* pages = p.page_table + (size_t)b * p.max_pages + pg_begin;
-    // One round of global loads: the parent array goes to shared memory (the ancestor walks below
-    // would otherwise be chains of dependent global loads), and the page ids of this slice are
-    // checked before the TMA warp uses them as coordinates.
-    if (tid == 0) s_flag = 0;
-    if (tid < SAGE_MAX_NODES) s_parent[tid] = (tid < N) ? p.parent[n0 + tid] : -1;
-    bool bad_page = false;
-    for (int j = tid; j < ns; j += kAttnThreads) {
-        const int id = pages[j];
-        if (id < 0 || id >= p.n_pages) bad_page = true;
-    }
-    __syncthreads();
-    if (bad_page) s_flag = 2;
-    if (tid < SAGE_MAX_NODES) {
-        uint64_t a = 0;
-        if (tid < N) {
-            bool bad = false;
-            a = ancestor_bits(s_parent, N, tid, &bad);
-            if (bad) { s_flag = 1; a = 1ull << tid; }
+    // ---- this gang's range of steps (warp 0 computes, everybody reads)
+    if (warp == 0) {
+        int err = 0;
+        const int Wb = steps_per_head(p, lane, &err);
+        if (err) report_status(p.status, err);
+        const long long W = (long long)p.n_layers * p.Hkv * Wb;
+        long long begin = 0, end = 0;
+        int lg = 0, b = 0, s0 = 0;
+        if (W > 0) {
+            const int n_act = active_gangs(W, p.n_gangs);
+            if (gang < n_act) {
+                begin = gang_begin(W, n_act, gang);
+                end = gang_begin(W, n_act, gang + 1);
+            }
+            if (end > begin) {
+                lg = (int)(begin / Wb);
+                locate(p, lane, (int)(begin % Wb), &b, &s0);
+            }
         }
-        s_anc[tid] = a;
+        if (lane == 0) {
+            sh->range_begin = begin; sh->range_end = end;
+            sh->first_lg = lg; sh->first_b = b; sh->first_s0 = s0;
+        }
     }
     __syncthreads();
-    if (s_flag) {
-        if (tid == 0) report_status(p.status, s_flag == 1 ? SAGE_STATUS_BAD_TREE : SAGE_STATUS_BAD_PAGE);
-        return;
-    }
+    if (sh->range_end <= sh->range_begin) return;       // uniform: nothing to do, nothing allocated yet
 
-    // ---- set-up: barriers, TMEM, Q tiles
+    // ---- set-up: barriers, TMEM
     if (tid == 0) {
-        for (int i = 0; i < kStages; ++i) {
-            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], n_rtiles);   // one release per MMA warp
-            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], n_rtiles);
-        }
+        for (int i = 0; i < kRing; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_done[i], 1); }
         for (int t = 0; t < 2; ++t) {
-            for (int x = 0; x < 2; ++x) { mbar_init(&bars->s_full[t][x], 1); mbar_init(&bars->p_full[t][x], 4); }
-            mbar_init(&bars->pv_done[t], 1);
-            mbar_init(&bars->o_full[t], 1);
+            mbar_init(&sh->s_full[t], 1);
+            mbar_init(&sh->p_full[t], 4);               // one arrival per softmax warp
+            mbar_init(&sh->o_full[t], 1);
         }
-        mbar_init(&bars->q_ready, 8);
-        bars->abort = 0;
+        mbar_init(&sh->q_free, 1);
+        mbar_init(&sh->drain, 1);
+        mbar_init(&sh->q_ready, 1);
+        sh->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&bars->tmem_base)), "r"(512) : "memory");
+                     ::"r"(smem_u32(&sh->tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // From here the TMA producer streams K/V while the softmax warps stage the query tiles.
-    if (warp < 8) {
-        // Q rows -> K-major 128B-swizzled tiles; rows past M are zero.  Eight 16-byte loads are in
-        // flight per thread before the first store (the loads are latency-bound otherwise).
-        for (int c0 = tid; c0 < n_rtiles * kRowTile * 16; c0 += 256 * 8) {
-            uint4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int c = c0 + u * 256;
-                const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
-                const int R = rpair * kRowsPerCta + t * kRowTile + r;
-                v[u] = make_uint4(0, 0, 0, 0);
-                if (R < M) {
-                    const size_t row = ((size_t)layer * p.sum_nodes + n0 + R / p.G) * p.Hq + g * p.G + R % p.G;
-                    v[u] = *reinterpret_cast<const uint4*>(p.q + row * kHeadDim + ch * 8);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int c = c0 + u * 256;
-                const int t = c / (kRowTile * 16), r = (c / 16) % kRowTile, ch = c % 16;
-                const int half = ch >> 3, cc = ch & 7;
-                *reinterpret_cast<uint4*>(sQ + t * kQTileBytes + half * kQHalfBytes + r * 128 + ((cc ^ (r & 7)) << 4)) = v[u];
-            }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA unit
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->q_ready);
-    }
-    const uint32_t tmem = bars->tmem_base;
+    const uint32_t tmem = sh->tmem_base;
 
+    // Registers move from the copy / MMA warpgroup (which needs few) to the softmax warpgroups:
+    // 4 warps give up 168 - 72 registers per thread, 8 warps take 216 - 168 each.
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 8) {
         // =========================== TMA producer ===========================
         if (lane == 0) {
-            int issued_k = 0, issued_v = 0;
-            for (int j = 0; j < ns; ++j) {
-                const int slot = j % kStages, use = j / kStages;
-                const int c2 = pages[j] * p.Hkv + g;
-                if (use > 0 && !mbar_wait(&bars->k_empty[slot], (use - 1) & 1, bars, p.status)) break;
-                mbar_expect_tx(&bars->k_full[slot], kPageBytes);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_4d(smem_u32(sK + slot * kPageBytes + h * kPageHalfBytes), &kmap, h * 64, 0, c2, layer,
-                                &bars->k_full[slot]);
-                issued_k = j + 1;
-                if (use > 0 && !mbar_wait(&bars->v_empty[slot], (use - 1) & 1, bars, p.status)) break;
-                mbar_expect_tx(&bars->v_full[slot], kPageBytes);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_4d(smem_u32(sV + slot * kPageBytes + h * kPageHalfBytes), &vmap, h * 64, 0, c2, layer,
-                                &bars->v_full[slot]);
-                issued_v = j + 1;
+            SegIter it;
+            it.init(sh);
+            Seg sg;
+            // A segment of n steps takes n + 1 ring steps: ring step i carries the K tile of step s0 + i
+            // (i < n) and the V tile of step s0 + i - 1 (i > 0), which is what the MMA warp consumes together
+            // ([P V of the step before, scores of this step]); both land on one barrier.
+            int rc = 0, kc = 0, vc = 0, nq = 0;          // ring steps, K tiles, V tiles, query loads issued so far
+            bool ok = !p.producer_off;
+            while (ok && it.next(p, sg)) {
+                if (member >= sg.rp) continue;
+                const int M = sg.N * p.G;
+                const int n_rt = (M - member * kRowsPerCta > kRowTile) ? 2 : 1;
+                const int32_t* pages = p.page_table + (size_t)sg.b * p.max_pages;
+                const int n_pages_seq = (sg.L + sg.N + kPageSize - 1) / kPageSize;
+                const int n = sg.s1 - sg.s0;
+                int ids_prev[2] = {0, 0}, npg_prev = 0;
+                for (int i = 0; i <= n; ++i) {
+                    const int j = sg.s0 + i;
+                    // page ids of step j (checked: they become TMA coordinates)
+                    int ids[2] = {0, 0}, npg = 0;
+                    if (i < n) {
+                        npg = (2 * j + 1 < n_pages_seq) ? 2 : 1;
+                        for (int pi = 0; pi < npg; ++pi) {
+                            ids[pi] = pages[2 * j + pi];
+                            if (ids[pi] < 0 || ids[pi] >= p.n_pages) {
+                                report_status(p.status, SAGE_STATUS_BAD_PAGE);
+                                ids[pi] = 0;
+                            }
+                        }
+                    }
+                    // the tiles that ring step rc - 2 used are free once its MMAs have finished
+                    if (rc >= 2 && !mbar_wait(&sh->kv_done[(rc - 2) % kRing], ((rc - 2) / kRing) & 1, sh, p)) { ok = false; break; }
+                    uint64_t* full = &sh->kv_full[rc % kRing];
+                    mbar_expect_tx(full, (npg + (i > 0 ? npg_prev : 0)) * 2 * kPageHalfBytes);
+                    if (i < n) {
+                        const int kslot = kc % kKStages;
+                        for (int pi = 0; pi < npg; ++pi)
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_4d(smem_u32(sK + kslot * kTileBytes + h * kTileHalfBytes + pi * kPageHalfBytes), &kmap,
+                                            h * 64, 0, ids[pi] * p.Hkv + sg.g, sg.layer, full);
+                        ++kc;
+                    }
+                    if (i > 0) {
+                        const int vslot = vc % kVStages;
+                        for (int pi = 0; pi < npg_prev; ++pi)
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_4d(smem_u32(sV + vslot * kTileBytes + h * kTileHalfBytes + pi * kPageHalfBytes), &vmap,
+                                            h * 64, 0, ids_prev[pi] * p.Hkv + sg.g, sg.layer, full);
+                        ++vc;
+                    }
+                    ++rc;
+                    if (i == 0) {
+                        // the segment's query tiles, once the previous segment's score MMAs have read theirs
+                        if (nq > 0 && !mbar_wait(&sh->q_free, (nq - 1) & 1, sh, p)) { ok = false; break; }
+                        mbar_expect_tx(&sh->q_ready, n_rt * kQTileBytes);
+                        for (int t = 0; t < n_rt; ++t)
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_5d(smem_u32(sQ + t * kQTileBytes + h * kQHalfBytes), &qmap, h * 64, 0, sg.g,
+                                            sg.n0 + (member * kRowsPerCta + t * kRowTile) / p.G, sg.layer, &sh->q_ready);
+                        ++nq;
+                    }
+                    ids_prev[0] = ids[0]; ids_prev[1] = ids[1]; npg_prev = npg;
+                }
             }
-            if (bars->abort) {
+            if (sh->abort) {
                 // drain: every issued copy must land before the CTA may exit
-                for (int n = max(0, issued_k - kStages); n < issued_k; ++n) {
-                    const long long t0 = clock64();
-                    while (!mbar_try(&bars->k_full[n % kStages], (n / kStages) & 1) && clock64() - t0 < kWaitCycles) {}
-                }
-                for (int n = max(0, issued_v - kStages); n < issued_v; ++n) {
-                    const long long t0 = clock64();
-                    while (!mbar_try(&bars->v_full[n % kStages], (n / kStages) & 1) && clock64() - t0 < kWaitCycles) {}
-                }
+                for (int n = max(0, rc - 2); n < rc; ++n)
+                    mbar_wait_quiet(&sh->kv_full[n % kRing], (n / kRing) & 1, p.wait_cycles);
+                if (nq > 0) mbar_wait_quiet(&sh->q_ready, (nq - 1) & 1, p.wait_cycles);
             }
         }
-    } else if (warp >= 9) {
-        // =========================== MMA issuers: warp 9 -> row tile 0, warp 10 -> row tile 1 ===========================
-        // Broadcasts from lane 0 tell the compiler that these values are warp-uniform, so that the
-        // descriptor arithmetic and the loop control below can stay in the uniform datapath.
-        const int t = __shfl_sync(0xffffffffu, warp - 9, 0);
-        const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
-        const int ns = __shfl_sync(0xffffffffu, max(0, pg_end - pg_begin), 0);
-        const int n_rtiles = __shfl_sync(0xffffffffu, (M - rpair * kRowsPerCta > kRowTile) ? 2 : 1, 0);
-        const int first_pos = __shfl_sync(0xffffffffu, pg_begin * kPageSize, 0);
-        const int T = __shfl_sync(0xffffffffu, L + N, 0);
-        const bool leader = elect_one();
-        // lane 0 polls, the result is broadcast so that the warp never diverges on a wait
-        auto wait_all = [&](uint64_t* bar, uint32_t parity) {
-            int r = 1;
-            if (lane == 0) r = mbar_wait(bar, parity, bars, p.status) ? 1 : 0;
-            return __shfl_sync(0xffffffffu, r, 0) != 0;
-        };
-        // descriptors differ only in their 14-bit start-address field (bytes >> 4); shared memory ends below 256 KB
-        const uint64_t dq = make_desc(smem_u32(sQ) + t * kQTileBytes, 16, 1024);
-        const uint64_t dk = make_desc(smem_u32(sK), 16, 1024);
-        const uint64_t dv = make_desc(smem_u32(sV), kPageHalfBytes, 1024);
-        const uint32_t s_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
-        auto issue_qk = [&](int x, int slot) {
-            // S_t,x = Q_t K^T: 8 steps of K = 16 over d = 128 (4 per 64-wide half)
-            const uint64_t dks = dk + (uint64_t)((slot * kPageBytes) >> 4);
-            const uint32_t d = s_tmem + x * 64;
-            mma_ss<false>(leader, d, dq, dks, kIdescQK);
+    } else if (warp == 9) {
+        // =========================== MMA issuer ===========================
+        // One thread issues for both row tiles, in blocks [P V of step j-1, scores of step j] per tile:
+        // a tile's block runs on the tensor pipe while the other tile's warpgroup is in its softmax, and
+        // the blocks of the two tiles never interleave (two issuers would finish both tiles' scores at
+        // the same moment and leave the pipe idle during both softmaxes).  The whole instruction stream
+        // sits in one single-thread region: a predicated branch around every MMA costs more issue time
+        // than the MMA takes to execute.
+        if (lane == 0) {
+            // descriptors differ only in their 14-bit start-address field (bytes >> 4); shared memory ends below 256 KB
+            const uint32_t dq = desc_lo(smem_u32(sQ), 16);
+            const uint32_t dk = desc_lo(smem_u32(sK), 16);
+            const uint32_t dv = desc_lo(smem_u32(sV), kTileHalfBytes);
+            auto issue_qk = [&](int t, int slot) {
+                // S_t = Q_t K^T: 8 slices of K = 16 over d = 128 (4 per 64-wide half)
+                const uint32_t dqt = dq + ((t * kQTileBytes) >> 4);
+                const uint32_t dks = dk + ((slot * kTileBytes) >> 4);
+                const uint32_t s_tmem = tmem + t * 128;
 #pragma unroll
-            for (int ks = 1; ks < 8; ++ks)
-                mma_ss<true>(leader, d, dq + (uint64_t)(((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4),
-                             dks + (uint64_t)(((ks >> 2) * kPageHalfBytes + (ks & 3) * 32) >> 4), kIdescQK);
-        };
-        auto issue_pv = [&](int x, int slot, bool first) {
-            // O_t += P_t,x V: 4 steps of K = 16 keys; P in TMEM (8 columns per step), V MN-major
-            const uint64_t dvs = dv + (uint64_t)((slot * kPageBytes) >> 4);
-            const uint32_t a = s_tmem + x * 64;
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ss(s_tmem, dqt + (((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4),
+                           dks + (((ks >> 2) * kTileHalfBytes + (ks & 3) * 32) >> 4), kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
+            };
+            auto issue_pv = [&](int t, int slot, bool first) {
+                // O_t += P_t V: 8 slices of K = 16 keys; P in TMEM (8 columns per slice), V MN-major
+                const uint32_t dvs = dv + ((slot * kTileBytes) >> 4);
+                const uint32_t s_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                mma_ts(leader, o_tmem, a + ks * 8, dvs + (uint64_t)((ks * 2048) >> 4), kIdescPV, (!first || ks > 0) ? 1u : 0u);
-        };
-        bool ok = ns > 0 && t < n_rtiles;
-        if (ok) ok = wait_all(&bars->q_ready, 0);
-        // prologue: scores of the first two pages
-        for (int j = 0; ok && j < min(2, ns); ++j) {
-            ok = wait_all(&bars->k_full[j], 0);
-            if (!ok) break;
-            tc_fence_after();
-            issue_qk(j, j);
-            tc_commit(leader, &bars->s_full[t][j]);
-            tc_commit(leader, &bars->k_empty[j]);
-        }
-        // The V page of step j and the K page of step j+2 are looked up one step ahead (`stage_inputs`),
-        // while the softmax of the previous page is still running, so that only the wait for the
-        // probabilities sits between the softmax and the MMAs that depend on it.
-        auto stage_inputs = [&](int j) -> bool {
-            if (j >= ns) return true;
-            const int vslot = j % kStages;
-            if (!wait_all(&bars->v_full[vslot], (j / kStages) & 1)) return false;
-            const int valid = min(kPageSize, T - first_pos - j * kPageSize);
-            if (valid < kPageSize) {
-                // rows past the end of the sequence may hold anything: zero them so that 0 * V stays 0
-                // (both MMA warps write the same zeros; each orders its own writes before its own MMAs)
-                uint8_t* vb = sV + vslot * kPageBytes;
-                for (int c = lane; c < (kPageSize - valid) * 16; c += 32) {
-                    const int r = valid + c / 16, ch = c % 16;
-                    *reinterpret_cast<uint4*>(vb + (ch >> 3) * kPageHalfBytes + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(o_tmem, s_tmem + ks * 8, dvs + ((ks * 2048) >> 4), kDescHi, kIdescPV, (first && ks == 0) ? 0u : 1u);
+            };
+            SegIter it;
+            it.init(sh);
+            Seg sg;
+            int rc = 0, kc = 0, vc = 0, nq = 0;             // ring steps, K tiles, V tiles consumed; segments started
+            int np[2] = {0, 0};                             // steps of each row tile whose probabilities were consumed
+            bool ok = true;
+            // Every synchronisation instruction costs this thread a couple of hundred clocks, during which
+            // at most a few queued MMAs keep the pipe busy: the loop holds as few of them as the protocol
+            // allows (one wait and one commit per ring step for the tiles, one of each per row tile).
+            while (ok && it.next(p, sg)) {
+                if (member >= sg.rp) continue;
+                const int n_rt = (sg.N * p.G - member * kRowsPerCta > kRowTile) ? 2 : 1;
+                const int s0 = sg.s0, s1 = sg.s1;
+                ok = mbar_wait(&sh->q_ready, nq & 1, sh, p);
+                ++nq;
+                // ring step: the P V products of step j - 1 (when j > s0) and the scores of step j (when j < s1)
+                for (int j = s0; ok && j <= s1; ++j) {
+                    ok = mbar_wait(&sh->kv_full[rc % kRing], (rc / kRing) & 1, sh, p);
+                    if (!ok) break;
+                    const int kslot = kc % kKStages, vslot = vc % kVStages;
+                    if (j < s1) ++kc;
+                    if (j > s0) ++vc;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (t < n_rt) {
+                            if (j > s0) {
+                                // (the warpgroup zeroed the V rows past the end of the sequence before it arrived)
+                                ok = mbar_wait(&sh->p_full[t], np[t] & 1, sh, p);
+                                if (!ok) break;
+                                ++np[t];
+                                tc_fence_after();
+                                issue_pv(t, vslot, j - 1 == s0);
+                                if (j == s1) tc_commit(true, &sh->o_full[t]);   // every MMA of this tile's segment has been issued
+                            }
+                            if (j < s1) {
+                                issue_qk(t, kslot);
+                                tc_commit(true, &sh->s_full[t]);
+                            }
+                        }
+                    }
+                    if (!ok) break;
+                    tc_commit(true, &sh->kv_done[rc % kRing]);
+                    ++rc;
+                    if (j == s1 - 1) tc_commit(true, &sh->q_free);          // the segment's last score MMAs read the query tiles
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
             }
-            const int jn = j + 2;
-            if (jn < ns && !wait_all(&bars->k_full[jn % kStages], (jn / kStages) & 1)) return false;
-            return true;
-        };
-        if (ok) ok = stage_inputs(0);
-        for (int j = 0; ok && j < ns; ++j) {
-            const int x = j & 1, vslot = j % kStages;
-            const int jn = j + 2, kslot = jn % kStages;
-            ok = wait_all(&bars->p_full[t][x], (j >> 1) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            issue_pv(x, vslot, j == 0);
-            tc_commit(leader, &bars->pv_done[t]);
-            tc_commit(leader, &bars->v_empty[vslot]);
-            if (jn < ns) {
-                // the scores of page j+2 reuse this S buffer: in pipe order after P V of page j
-                issue_qk(x, kslot);
-                tc_commit(leader, &bars->s_full[t][x]);
-                tc_commit(leader, &bars->k_empty[kslot]);
+            if (!ok) {
+                // abort: everything this thread has issued must retire before the TMEM and the tiles go away
+                tc_commit(true, &sh->drain);
+                mbar_wait_quiet(&sh->drain, 0, p.wait_cycles);
             }
-            ok = stage_inputs(j + 1);
         }
-        if (t < n_rtiles) tc_commit(leader, &bars->o_full[t]);     // arrives when every MMA of this tile has completed
         __syncwarp();
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== softmax warpgroups ===========================
         const int t = warp >> 2;                        // row tile of this warpgroup
         const int r = tid & 127;                        // row inside the tile == TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t s_taddr = tmem + lane_base + t * 128;
         const uint32_t o_taddr = tmem + lane_base + 256 + t * 128;
-        const int R = rpair * kRowsPerCta + t * kRowTile + r;
-        const bool row_ok = R < M;
-        const int node = row_ok ? R / p.G : 0;
-        const uint64_t anc = s_anc[node];
-        const bool warp_live = rpair * kRowsPerCta + t * kRowTile + (warp & 3) * 32 < M;
-        float m_ref = -INFINITY, l_sum = 0.f;
-        bool ok = (t < n_rtiles);
-        for (int j = 0; ok && j < ns; ++j) {
-            const int x = j & 1;
-            ok = mbar_wait(&bars->s_full[t][x], (j >> 1) & 1, bars, p.status);
-            if (!ok) break;
-            if (!warp_live) {
-                // none of this warp's 32 rows exists (ragged last tile): keep the barrier protocol
-                // going, leave the probabilities of these rows as they are; their outputs are never stored
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->p_full[t][x]);
-                continue;
+        SegIter it;
+        it.init(sh);
+        Seg sg;
+        int nsteps = 0, nseg = 0;                       // steps / segments this row tile has been through
+        int rc0 = 0, vc0 = 0;                           // ring steps / V tiles of the CTA before the current segment
+        bool ok = true;
+        while (ok && it.next(p, sg)) {
+            if (member >= sg.rp) continue;
+            const int M = sg.N * p.G;
+            const int rc_seg = rc0, vc_seg = vc0;       // this segment's first ring step / V tile
+            rc0 += sg.s1 - sg.s0 + 1;
+            vc0 += sg.s1 - sg.s0;
+            if (t == 1 && M - member * kRowsPerCta <= kRowTile) continue;
+            const int R = member * kRowsPerCta + t * kRowTile + r;
+            const bool row_ok = R < M;
+            const int node = row_ok ? R / p.G : 0;
+            const bool warp_live = member * kRowsPerCta + t * kRowTile + (warp & 3) * 32 < M;
+            uint64_t anc = 0;
+            if (sg.s1 * kStepKeys > sg.L && row_ok) {
+                // the segment reaches the tree part: this row's ancestor bitset (the G rows of a node
+                // walk the same parent chain, at most N - 1 cached loads deep)
+                bool bad = false;
+                anc = ancestor_bits(p.parent + sg.n0, sg.N, node, &bad);
+                if (bad) { report_status(p.status, SAGE_STATUS_BAD_TREE); anc = 1ull << node; }
             }
-            tc_fence_after();
-            uint32_t sr[64];
-            tmem_ld32(s_taddr + x * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-            tmem_ld32(s_taddr + x * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-            tmem_wait_ld();
-            const int pos0 = (pg_begin + j) * kPageSize;
-            const bool masked = pos0 + kPageSize > L;
-            if (masked) {
-                // page reaches into the tree part (or past the end): apply the ancestor mask
-#pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const int jt = pos0 + i - L;                      // tree slot; < 0 = prefix
-                    const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
-                    if (!vis) sr[i] = 0xff800000u;                    // -inf
-                }
-            }
-            // row max: eight independent chains of three-input max
-            float mx8[8];
-#pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) {
-                float mq = max3(__uint_as_float(sr[q8 * 8]), __uint_as_float(sr[q8 * 8 + 1]), __uint_as_float(sr[q8 * 8 + 2]));
-                mq = max3(mq, __uint_as_float(sr[q8 * 8 + 3]), __uint_as_float(sr[q8 * 8 + 4]));
-                mq = max3(mq, __uint_as_float(sr[q8 * 8 + 5]), __uint_as_float(sr[q8 * 8 + 6]));
-                mx8[q8] = fmaxf(mq, __uint_as_float(sr[q8 * 8 + 7]));
-            }
-            const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), fmaxf(max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-            const float m_cand = mx * p.scale_log2;
-            // lazy rescale: move the reference only when the row max grew by more than 2^8
-            const bool grow = m_cand > m_ref + 8.0f;
-            float alpha = 1.0f;
-            if (grow) {
-                alpha = fast_exp2(m_ref - m_cand);          // 0 when m_ref was -inf
-                m_ref = m_cand;
-            }
-            const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                // O_t *= alpha, once the P V product of page j-1 has finished
-                ok = mbar_wait(&bars->pv_done[t], (j - 1) & 1, bars, p.status);
-                ok = __all_sync(0xffffffffu, ok);
+            float m_ref = -INFINITY, l_sum = 0.f;
+            for (int j = sg.s0; j < sg.s1; ++j) {
+                ok = mbar_wait(&sh->s_full[t], nsteps & 1, sh, p);
                 if (!ok) break;
+                const int valid = sg.L + sg.N - j * kStepKeys;      // keys of this step that exist
+                if (valid < kStepKeys) {
+                    // V rows past the end of the sequence may hold anything (a missing second page was not even
+                    // copied): zero them so that 0 * V stays 0.  Each warp of the warpgroup takes a quarter of
+                    // the rows (both warpgroups write the same zeros); the writes are ordered before this
+                    // warp's arrival, which the P V product waits for.  The V tile of step j lands with ring
+                    // step j - s0 + 1 of the segment.
+                    const int rcv = rc_seg + (j - sg.s0) + 1;
+                    ok = mbar_wait(&sh->kv_full[rcv % kRing], (rcv / kRing) & 1, sh, p);
+                    if (!ok) break;
+                    uint8_t* vb = sV + ((vc_seg + (j - sg.s0)) % kVStages) * kTileBytes;
+                    for (int c = (warp & 3) * 32 + lane; c < (kStepKeys - valid) * 16; c += 128) {
+                        const int vr = valid + c / 16, ch = c % 16;
+                        *reinterpret_cast<uint4*>(vb + (ch >> 3) * kTileHalfBytes + vr * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                if (!warp_live) {
+                    // none of this warp's 32 rows exists (ragged last tile): keep the barrier protocol
+                    // going, leave the probabilities of these rows as they are; their outputs are never stored
+                    ++nsteps;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh->p_full[t]);
+                    continue;
+                }
                 tc_fence_after();
-                rescale_o_rows(o_taddr, alpha);
+                const int pos0 = j * kStepKeys;
+                const bool masked = pos0 + kStepKeys > sg.L;     // reaches into the tree part (or past the end)
+                uint32_t sr[128];
+                load_scores(s_taddr, sr);
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) mask_chunk(sr + 32 * c, pos0 + 32 * c, sg.L, sg.N, anc);
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) max_chunk(sr + 32 * c, mx);
+                // lazy rescale: the reference moves only when the row max grew by more than 2^8 over it
+                const float m_cand = mx * p.scale_log2;
+                const bool grow = m_cand > m_ref + 8.0f;
+                float alpha = 1.0f;
+                if (grow) {
+                    alpha = fast_exp2(m_ref - m_cand);              // 0 when m_ref was -inf
+                    m_ref = m_cand;
+                }
+                // O_t *= alpha.  The P V product of the step before has finished: the scores of this step were
+                // issued after it, and their completion is what this warp waited for above.
+                if (j > sg.s0 && __any_sync(0xffffffffu, grow)) rescale_o_rows(o_taddr, alpha);
+                const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                // probabilities, packed to bf16 in place: chunk c (32 scores) leaves its 16 words at sr[16c ..]
+                uint64_t acc[2] = {0ull, 0ull};
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) exp_chunk<0>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);   // may hold -inf
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) exp_chunk<SAGE_EXP2_FMA_PAIRS>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);
+                }
+                float sum_a, sum_b;
+                f2_unpack(f2_add(acc[0], acc[1]), sum_a, sum_b);
+                l_sum = l_sum * alpha + (sum_a + sum_b);
+                uint32_t* pk = sr;
+                tmem_st32(s_taddr, pk);                 // P over the first 64 columns of S_t
+                tmem_st32(s_taddr + 32, pk + 32);
+                tmem_wait_st();
+                tc_fence_before();
+                ++nsteps;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->p_full[t]);
             }
-            float sum;
-            if (masked) sum = softmax_half<0>(sr, p.scale_log2, neg_ref);     // may hold -inf
-            else sum = softmax_half<SAGE_EXP2_FMA_PAIRS>(sr, p.scale_log2, neg_ref);
-            tmem_st32(s_taddr + x * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));   // P over the first 32 columns of this S buffer
-            l_sum = l_sum * alpha + sum;
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->p_full[t][x]);
-        }
-        // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
-        if (t < n_rtiles) {
-            if (ns > 0 && ok) ok = mbar_wait(&bars->o_full[t], 0, bars, p.status);
-            if (ok) tc_fence_after();
-            const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
-            const size_t row = (size_t)(n0 + node) * p.Hq + g * p.G + (row_ok ? R % p.G : 0);
+            if (!ok) break;
+            // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
+            ok = mbar_wait(&sh->o_full[t], nseg & 1, sh, p);
+            ++nseg;
+            if (!ok) break;
+            tc_fence_after();
+            const bool whole = (sg.s0 == 0 && sg.s1 == sg.steps);
             const float inv = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
             float* po = nullptr;
             __nv_bfloat16* oo = nullptr;
-            if (p.n_splits == 1) {
-                oo = p.out + ((size_t)layer * rows_total + row) * kHeadDim;
+            if (whole) {
+                const size_t row = (size_t)(sg.n0 + node) * p.Hq + sg.g * p.G + (row_ok ? R % p.G : 0);
+                oo = p.out + ((size_t)sg.layer * p.sum_nodes * p.Hq + row) * kHeadDim;
             } else {
-                const size_t pr = ((size_t)layer * p.n_splits + split) * rows_total + row;
+                const size_t pr = (((size_t)gang * 2 + (sg.at_range_begin ? 0 : 1)) * p.n_rp + member) * kRowsPerCta +
+                                  t * kRowTile + r;
                 po = p.part_o + pr * kHeadDim;
-                if (row_ok && ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = (ns > 0) ? l_sum : 0.f; }
+                if (row_ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = l_sum; }
             }
+            if (warp_live) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t orr[32];
-                if (ns > 0 && ok) {
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t orr[32];
                     tmem_ld32(o_taddr + c * 32, orr);
                     tmem_wait_ld();
-                } else {
+                    if (row_ok) {
+                        if (oo) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) orr[i] = 0u;
-                }
-                if (row_ok && ok) {
-                    if (oo) {
+                            for (int i = 0; i < 4; ++i) {
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+                                *reinterpret_cast<uint4*>(oo + c * 32 + i * 8) = v;
+                            }
+                        } else {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint4 v;
-                            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-                            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-                            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-                            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4*>(oo + c * 32 + i * 8) = v;
+                            for (int i = 0; i < 8; ++i)
+                                *reinterpret_cast<uint4*>(po + c * 32 + i * 4) =
+                                    make_uint4(orr[4 * i], orr[4 * i + 1], orr[4 * i + 2], orr[4 * i + 3]);
                         }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            *reinterpret_cast<uint4*>(po + c * 32 + i * 4) =
-                                make_uint4(orr[4 * i], orr[4 * i + 1], orr[4 * i + 2], orr[4 * i + 3]);
                     }
                 }
             }
+            tc_fence_before();                          // the next segment's first P V overwrites O_t
         }
     }
     // ---- teardown: every role is past its last TMEM access
@@ -677,64 +862,78 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     }
 }
 
-// Split-K merge: one warp per (layer, node, head) row.  Lanes first reduce (m, l) over
-// the slices with shuffles, then each lane combines its four output columns.
-__global__ void attention_merge_kernel(AttnParams p) {
-    const int warps = blockDim.x >> 5;
-    const size_t rows_total = (size_t)p.sum_nodes * p.Hq;
-    const size_t row = (size_t)blockIdx.x * warps + (threadIdx.x >> 5);
-    const int layer = blockIdx.y;
-    const int lane = threadIdx.x & 31;
-    if (row >= rows_total) return;
-    const int node = (int)(row / p.Hq);
-    if (node >= p.node_offsets[p.batch]) return;       // rows past the live nodes were never written
-    float m = -INFINITY, l = 0.f;
-    if (lane < p.n_splits) {
-        const size_t r = ((size_t)layer * p.n_splits + lane) * rows_total + row;
-        m = p.part_ml[r * 2];
-        l = p.part_ml[r * 2 + 1];
+// Merge of the items that a range boundary cut into segments.  Only a boundary between two gangs'
+// ranges can cut an item, so the grid is (x = boundary, y = 32-row chunk): the block finds the item
+// its boundary falls into, leaves if the boundary coincides with the item's start or if an earlier
+// boundary already lies inside the same item (that block does the work), and otherwise combines the
+// item's segments: which gangs hold them, and in which of their two partial slots, follows from
+// the positions alone.
+__global__ void __launch_bounds__(256) attention_merge_kernel(AttnParams p) {
+    __shared__ int s_Wb, s_b, s_s0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_cut = blockIdx.x + 1;                   // boundary between gang k_cut - 1 and gang k_cut
+    if (warp == 0) {
+        int err = 0, b = 0, s0 = 0;
+        const int Wb = steps_per_head(p, lane, &err);
+        if (Wb > 0) {
+            const long long W = (long long)p.n_layers * p.Hkv * Wb;
+            const int n_act = active_gangs(W, p.n_gangs);
+            if (k_cut < n_act) locate(p, lane, (int)(gang_begin(W, n_act, k_cut) % Wb), &b, &s0);
+        }
+        if (lane == 0) { s_Wb = Wb; s_b = b; s_s0 = s0; }
     }
-    float mx = (l > 0.f) ? m : -INFINITY;
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    const float w = (l > 0.f) ? exp2f(m - mx) : 0.f;   // weight of this lane's slice
-    float lsum = l * w;
-    for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < p.n_splits; ++s) {
-        const float ws = __shfl_sync(0xffffffffu, w, s);
-        if (ws == 0.f) continue;
-        const size_t r = ((size_t)layer * p.n_splits + s) * rows_total + row;
-        const float4 v = reinterpret_cast<const float4*>(p.part_o + r * kHeadDim)[lane];
-        acc.x = fmaf(ws, v.x, acc.x); acc.y = fmaf(ws, v.y, acc.y);
-        acc.z = fmaf(ws, v.z, acc.z); acc.w = fmaf(ws, v.w, acc.w);
+    __syncthreads();
+    const int Wb = s_Wb;
+    if (Wb <= 0) return;
+    const long long W = (long long)p.n_layers * p.Hkv * Wb;
+    const int n_act = active_gangs(W, p.n_gangs);
+    if (k_cut >= n_act || s_s0 == 0) return;            // no such boundary, or it falls between two items
+    const long long cut = gang_begin(W, n_act, k_cut);
+    const int lg = (int)(cut / Wb), b = s_b;
+    int err = 0;
+    const Item it = load_item(p, b, &err);
+    const long long a = cut - s_s0;                     // position of the item's first step
+    const int k_first = gang_of(W, n_act, a), k_last = gang_of(W, n_act, a + it.steps - 1);
+    if (k_first != k_cut - 1) return;                   // an earlier boundary cuts the same item
+    const bool first_mid_range = (a != gang_begin(W, n_act, k_first));
+    const int M = it.N * p.G;
+    const int layer = lg / p.Hkv, g = lg % p.Hkv;
+    for (int i = 0; i < 4; ++i) {
+        const int R = blockIdx.y * 32 + warp * 4 + i;
+        if (R >= M) break;
+        const int member = R / kRowsPerCta, Rl = R % kRowsPerCta;
+        auto slot_row = [&](int k) -> size_t {
+            const int slot = (k == k_first && first_mid_range) ? 1 : 0;
+            return (((size_t)k * 2 + slot) * p.n_rp + member) * kRowsPerCta + Rl;
+        };
+        float mx = -INFINITY;
+        for (int k = k_first + lane; k <= k_last; k += 32) {
+            const size_t pr = slot_row(k);
+            if (p.part_ml[pr * 2 + 1] > 0.f) mx = fmaxf(mx, p.part_ml[pr * 2]);
+        }
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float lsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = k_first; k <= k_last; ++k) {
+            const size_t pr = slot_row(k);
+            const float l = p.part_ml[pr * 2 + 1];
+            if (!(l > 0.f)) continue;
+            const float w = exp2f(p.part_ml[pr * 2] - mx);
+            lsum = fmaf(l, w, lsum);
+            const float4 v = reinterpret_cast<const float4*>(p.part_o + pr * kHeadDim)[lane];
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+            acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        }
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        uint2 packed;
+        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+        const size_t row = (size_t)(it.n0 + R / p.G) * p.Hq + g * p.G + R % p.G;
+        reinterpret_cast<uint2*>(p.out + ((size_t)layer * p.sum_nodes * p.Hq + row) * kHeadDim)[lane] = packed;
     }
-    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-    uint2 packed;
-    packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-    packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-    reinterpret_cast<uint2*>(p.out + ((size_t)layer * rows_total + row) * kHeadDim)[lane] = packed;
 }
 
-static int pick_splits(int n_layers, int batch, int n_kv_heads, int G, int max_pages) {
-    // One CTA is resident per SM.  Take the smallest slice count whose CTA count fills whole
-    // waves of 148 SMs to >= 90 % (else the best one), keeping >= 4 pages per slice (short contexts are latency-bound:
-    // more, shorter slices beat fewer CTAs with longer loops; measured at 2k context).
-    const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
-    const long base = (long)n_layers * batch * n_kv_heads * row_pairs;
-    int s_max = max_pages / 4;
-    if (s_max > 32) s_max = 32;
-    if (s_max < 1) s_max = 1;
-    int best = 1;
-    double best_eff = 0.0;
-    for (int s = 1; s <= s_max; ++s) {
-        const long ctas = base * s;
-        const double eff = (double)ctas / (148.0 * ((ctas + 147) / 148));
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
-        if (eff >= 0.9) { best = s; break; }
-    }
-    return best;
-}
-
+// ---- host side ------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -751,22 +950,99 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Tensor maps depend only on (base pointer, shape); a serving loop calls with the same few buffers
+// over and over, so the last few encodings are kept.
+struct MapKey {
+    const void* base;
+    long long a, b, c, d;
+    int kind;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && a == o.a && b == o.b && c == o.c && d == o.d && kind == o.kind;
+    }
+};
+constexpr int kMapCache = 16;
+static std::mutex g_map_mu;
+static MapKey g_map_key[kMapCache];
+static CUtensorMap g_map_val[kMapCache];
+static int g_map_used = 0, g_map_next = 0;
+
+template <typename Make>
+static bool cached_map(CUtensorMap* out, const MapKey& key, Make make) {
+    std::lock_guard<std::mutex> lock(g_map_mu);
+    for (int i = 0; i < g_map_used; ++i)
+        if (g_map_key[i] == key) { *out = g_map_val[i]; return true; }
+    if (!make(out)) return false;
+    g_map_key[g_map_next] = key;
+    g_map_val[g_map_next] = *out;
+    g_map_next = (g_map_next + 1) % kMapCache;
+    if (g_map_used < kMapCache) ++g_map_used;
+    return true;
+}
+
 // Pool viewed as [layer][page*Hkv + head][slot][d]; one box = one 64-wide d-half of one (page, head).
 static bool make_pool_map(CUtensorMap* map, const void* pool, int n_layers, int n_pages, int n_kv_heads,
                           int64_t layer_stride_elems) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t page_head_bytes = (cuuint64_t)kPageSize * kHeadDim * 2;
-    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)kPageSize, (cuuint64_t)n_pages * n_kv_heads,
-                          (cuuint64_t)n_layers};
-    cuuint64_t layer_bytes = n_layers > 1 ? (cuuint64_t)layer_stride_elems * 2 : dims[2] * page_head_bytes;
-    cuuint64_t strides[3] = {(cuuint64_t)kHeadDim * 2, page_head_bytes, layer_bytes};
-    cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const MapKey key{pool, n_layers, n_pages, n_kv_heads, layer_stride_elems, 0};
+    return cached_map(map, key, [&](CUtensorMap* m) {
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return false;
+        const cuuint64_t page_head_bytes = (cuuint64_t)kPageSize * kHeadDim * 2;
+        cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)kPageSize, (cuuint64_t)n_pages * n_kv_heads,
+                              (cuuint64_t)n_layers};
+        cuuint64_t layer_bytes = n_layers > 1 ? (cuuint64_t)layer_stride_elems * 2 : dims[2] * page_head_bytes;
+        cuuint64_t strides[3] = {(cuuint64_t)kHeadDim * 2, page_head_bytes, layer_bytes};
+        cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
+
+// Queries viewed as [layer][node][kv head][head in group][d]; one box = one 64-wide d-half of the
+// 128 query rows (128/G nodes x G heads) of a row tile.  Nodes past sum_nodes read as zero.
+static bool make_q_map(CUtensorMap* map, const void* q, int n_layers, int sum_nodes, int n_kv_heads, int G) {
+    const MapKey key{q, n_layers, sum_nodes, n_kv_heads, G, 1};
+    return cached_map(map, key, [&](CUtensorMap* m) {
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return false;
+        const cuuint64_t row = (cuuint64_t)kHeadDim * 2;
+        cuuint64_t dims[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)G, (cuuint64_t)n_kv_heads, (cuuint64_t)sum_nodes,
+                              (cuuint64_t)n_layers};
+        cuuint64_t strides[4] = {row, row * G, row * G * n_kv_heads, row * G * n_kv_heads * sum_nodes};
+        cuuint32_t box[5] = {64, (cuuint32_t)G, 1, (cuuint32_t)(kRowTile / G), 1};
+        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
+}
+
+// One resident CTA per SM (148 when no device can be asked, e.g. a size query on a host without a GPU).
+static int resident_ctas() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            return 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+static int row_pairs(int sum_nodes, int G) {
+    const int n = sum_nodes < SAGE_MAX_NODES ? sum_nodes : SAGE_MAX_NODES;      // a tree has at most that many nodes
+    return (n * G + kRowsPerCta - 1) / kRowsPerCta;
+}
+
+static long long g_wait_cycles = kWaitCyclesDefault;
+static int g_producer_off = 0;
 
 }  // namespace sage
 
@@ -774,10 +1050,17 @@ using namespace sage;
 
 extern "C" size_t sage_tree_attention_workspace_size(int n_layers, int batch, int sum_nodes, int n_q_heads,
                                                      int n_kv_heads, int head_dim, int max_pages_per_seq) {
-    if (n_layers < 1 || batch < 1 || sum_nodes < 1 || n_q_heads < 1 || n_kv_heads < 1 || max_pages_per_seq < 1) return 0;
-    const int S = pick_splits(n_layers, batch, n_kv_heads, n_q_heads / n_kv_heads, max_pages_per_seq);
-    if (S == 1) return 16;
-    return (size_t)n_layers * S * sum_nodes * n_q_heads * (head_dim + 2) * sizeof(float);
+    if (n_layers < 1 || batch < 1 || sum_nodes < 1 || n_q_heads < 1 || n_kv_heads < 1 || max_pages_per_seq < 1 ||
+        n_q_heads % n_kv_heads)
+        return 0;
+    (void)head_dim;
+    // two partial slots (head and tail of its range) per resident CTA, independent of the problem size
+    return (size_t)resident_ctas() * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float);
+}
+
+extern "C" void sage_debug_attention_waits(long long wait_cycles, int producer_off) {
+    g_wait_cycles = wait_cycles > 0 ? wait_cycles : kWaitCyclesDefault;
+    g_producer_off = producer_off ? 1 : 0;
 }
 
 extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void* v_pool, int64_t layer_stride_elems,
@@ -795,29 +1078,33 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     if (n_q_heads % n_kv_heads) return SAGE_ERR_UNSUPPORTED;
     const int G = n_q_heads / n_kv_heads;
     if (G != 1 && G != 2 && G != 4 && G != 8) return SAGE_ERR_UNSUPPORTED;
-    if ((long)n_layers * batch * n_kv_heads > 65535) return SAGE_ERR_UNSUPPORTED;
+    if ((long long)n_layers * batch * n_kv_heads > 0x7fffffffll || max_pages_per_seq > (1 << 24)) return SAGE_ERR_UNSUPPORTED;
     if ((((uintptr_t)q | (uintptr_t)k_pool | (uintptr_t)v_pool | (uintptr_t)out) & 15) || (layer_stride_elems & 7))
         return SAGE_ERR_INVALID_ARG;
     if (n_layers > 1 && layer_stride_elems < (int64_t)n_pages * n_kv_heads * kPageSize * kHeadDim)
         return SAGE_ERR_INVALID_ARG;
     if (batch == 0) return SAGE_OK;
-    const int S = pick_splits(n_layers, batch, n_kv_heads, G, max_pages_per_seq);
     const size_t need = sage_tree_attention_workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads,
                                                            head_dim, max_pages_per_seq);
-    if (S > 1 && (!ws || ws_bytes < need || ((uintptr_t)ws & 15))) return SAGE_ERR_WORKSPACE;
+    if (!ws || ws_bytes < need || ((uintptr_t)ws & 15)) return SAGE_ERR_WORKSPACE;
+    const int n_ctas = resident_ctas();
     AttnParams p{};
-    p.q = (const __nv_bfloat16*)q;
+    p.n_rp = row_pairs(sum_nodes, G);
+    p.n_gangs = n_ctas / p.n_rp;
     p.out = (__nv_bfloat16*)out;
     p.part_o = (float*)ws;
-    p.part_ml = S > 1 ? (float*)ws + (size_t)n_layers * S * sum_nodes * n_q_heads * kHeadDim : nullptr;
+    p.part_ml = (float*)ws + (size_t)n_ctas * 2 * kRowsPerCta * kHeadDim;
     p.page_table = page_table; p.seq_len = seq_len; p.parent = parent; p.node_offsets = node_offsets;
     p.status = status;
     p.n_layers = n_layers; p.batch = batch; p.sum_nodes = sum_nodes; p.n_pages = n_pages;
-    p.max_pages = max_pages_per_seq; p.Hq = n_q_heads; p.Hkv = n_kv_heads; p.G = G; p.n_splits = S;
+    p.max_pages = max_pages_per_seq; p.Hq = n_q_heads; p.Hkv = n_kv_heads; p.G = G;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.wait_cycles = g_wait_cycles;
+    p.producer_off = g_producer_off;
 
-    CUtensorMap kmap, vmap;
-    if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
+    CUtensorMap qmap, kmap, vmap;
+    if (!make_q_map(&qmap, q, n_layers, sum_nodes, n_kv_heads, G) ||
+        !make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
         !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
         return SAGE_ERR_CUDA;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
@@ -830,12 +1117,9 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
             return SAGE_ERR_CUDA;
         attr_set[dev] = true;
     }
-    const int row_pairs = (SAGE_MAX_NODES * G + kRowsPerCta - 1) / kRowsPerCta;
-    dim3 grid(S, row_pairs, n_layers * batch * n_kv_heads);
-    tree_attention_kernel<<<grid, kAttnThreads, kSmemBytes, as_stream(stream)>>>(p, kmap, vmap);
-    if (S > 1) {
-        const size_t rows_total = (size_t)sum_nodes * n_q_heads;
-        dim3 mg((unsigned)((rows_total + 7) / 8), n_layers);
+    tree_attention_kernel<<<p.n_gangs * p.n_rp, kAttnThreads, kSmemBytes, as_stream(stream)>>>(p, qmap, kmap, vmap);
+    if (p.n_gangs > 1) {
+        dim3 mg((unsigned)(p.n_gangs - 1), (unsigned)((p.n_rp * kRowsPerCta + 31) / 32));
         attention_merge_kernel<<<mg, 256, 0, as_stream(stream)>>>(p);
     }
     return launch_status();

@@ -197,51 +197,57 @@ struct CompactParams {
     int32_t* status;
 };
 
+// Checks one sequence's accepted path and, when `src` / `dst` are given, turns it into element
+// offsets of the (page, head 0, slot) rows to move (-1 = row already in place).  Returns the
+// number of path entries, or 0 with *code set when the path or a page id is not valid: such a
+// sequence is left exactly as it is (nothing moves, its length does not advance).
+__device__ int plan_compaction(const CompactParams& p, int b, int64_t* src, int64_t* dst, int* code) {
+    const int L = p.seq_len[b];
+    int plen = p.path_len[b];
+    bool bad_path = (plen < 0 || plen > p.max_path || plen > SAGE_MAX_NODES || L < 0);
+    bool bad_page = false;
+    if (bad_path) plen = 0;
+    int prev = -1;
+    for (int j = 0; j < plen; ++j) {
+        const int node = p.path[(size_t)b * p.max_path + j];
+        int64_t so = -1, dofs = -1;
+        if (node <= prev || node < j || node >= SAGE_MAX_NODES || (j == 0 && node != 0)) {
+            bad_path = true;                       // a root path starts at 0 and visits increasing indices
+        } else if (node != j) {
+            const int s_pos = L + node, d_pos = L + j;
+            if (s_pos / kPageSize >= p.max_pages) {
+                bad_page = true;
+            } else {
+                const int sp = p.page_table[(size_t)b * p.max_pages + s_pos / kPageSize];
+                const int dp = p.page_table[(size_t)b * p.max_pages + d_pos / kPageSize];
+                if (sp < 0 || sp >= p.n_pages || dp < 0 || dp >= p.n_pages) {
+                    bad_page = true;
+                } else {
+                    so = ((int64_t)sp * p.n_kv_heads * kPageSize + s_pos % kPageSize) * kHeadDim;
+                    dofs = ((int64_t)dp * p.n_kv_heads * kPageSize + d_pos % kPageSize) * kHeadDim;
+                }
+            }
+        }
+        prev = node;
+        if (src) { src[j] = so; dst[j] = dofs; }
+    }
+    *code = bad_path ? SAGE_STATUS_BAD_PATH : (bad_page ? SAGE_STATUS_BAD_PAGE : 0);
+    return *code ? 0 : plen;
+}
+
 __global__ void __launch_bounds__(256) compact_kv_kernel(CompactParams p) {
     __shared__ int64_t s_src[SAGE_MAX_NODES];   // element offset of (page, head 0, slot) rows, -1 = skip
     __shared__ int64_t s_dst[SAGE_MAX_NODES];
     __shared__ int s_len;
     const int b = blockIdx.x;
     const int layer = blockIdx.y;
-    const int L = p.seq_len[b];
-    int plen = p.path_len[b];
     if (threadIdx.x == 0) {
-        bool bad_path = (plen < 0 || plen > p.max_path || plen > SAGE_MAX_NODES || L < 0);
-        bool bad_page = false;
-        if (bad_path) plen = 0;
-        int prev = -1;
-        for (int j = 0; j < plen; ++j) {
-            const int node = p.path[(size_t)b * p.max_path + j];
-            int64_t so = -1, dofs = -1;
-            if (node <= prev || node < j || node >= SAGE_MAX_NODES || (j == 0 && node != 0)) {
-                bad_path = true;                       // a root path starts at 0 and visits increasing indices
-            } else if (node != j) {
-                const int src = L + node, dst = L + j;
-                if (src / kPageSize >= p.max_pages) {
-                    bad_page = true;
-                } else {
-                    const int sp = p.page_table[(size_t)b * p.max_pages + src / kPageSize];
-                    const int dp = p.page_table[(size_t)b * p.max_pages + dst / kPageSize];
-                    if (sp < 0 || sp >= p.n_pages || dp < 0 || dp >= p.n_pages) {
-                        bad_page = true;
-                    } else {
-                        so = ((int64_t)sp * p.n_kv_heads * kPageSize + src % kPageSize) * kHeadDim;
-                        dofs = ((int64_t)dp * p.n_kv_heads * kPageSize + dst % kPageSize) * kHeadDim;
-                    }
-                }
-            }
-            prev = node;
-            s_src[j] = so;
-            s_dst[j] = dofs;
-        }
-        if (bad_path || bad_page) {                    // move nothing for this sequence
-            report_status(p.status, bad_path ? SAGE_STATUS_BAD_PATH : SAGE_STATUS_BAD_PAGE);
-            plen = 0;
-        }
-        s_len = plen;
+        int code = 0;
+        s_len = plan_compaction(p, b, s_src, s_dst, &code);
+        if (code) report_status(p.status, code);
     }
     __syncthreads();
-    plen = s_len;
+    const int plen = s_len;
     const int cols = p.n_kv_heads * 16;          // 16-byte chunks per token row across heads
     for (int c = threadIdx.x; c < 2 * cols; c += blockDim.x) {
         __nv_bfloat16* pool = (c < cols ? p.k_pool : p.v_pool) + (int64_t)layer * p.layer_stride;
@@ -263,11 +269,14 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(CompactParams p) {
     }
 }
 
-__global__ void advance_seq_len_kernel(int32_t* seq_len, const int32_t* path_len, int batch, int max_path) {
+// Runs after compact_kv_kernel (same stream): a sequence's length advances only when its path
+// passed the same checks, i.e. only when its rows were actually moved.
+__global__ void advance_seq_len_kernel(CompactParams p, int32_t* seq_len) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= batch) return;
-    const int pl = path_len[b];
-    if (pl >= 0 && pl <= max_path) seq_len[b] += pl;
+    if (b >= p.batch) return;
+    int code = 0;
+    const int plen = plan_compaction(p, b, nullptr, nullptr, &code);
+    if (!code) seq_len[b] += plen;
 }
 
 // ---------------------------------------------------------------------------
@@ -448,7 +457,7 @@ extern "C" int sage_compact_kv(void* k_pool, void* v_pool, int64_t layer_stride_
     CompactParams p{(__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, layer_stride_elems, n_layers, n_pages,
                     max_pages_per_seq, batch, max_path, n_kv_heads, page_table, seq_len, path, path_len, status};
     compact_kv_kernel<<<dim3(batch, n_layers), 256, 0, as_stream(stream)>>>(p);
-    advance_seq_len_kernel<<<(batch + 127) / 128, 128, 0, as_stream(stream)>>>(seq_len, path_len, batch, max_path);
+    advance_seq_len_kernel<<<(batch + 127) / 128, 128, 0, as_stream(stream)>>>(p, seq_len);
     return launch_status();
 }
 

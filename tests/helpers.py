@@ -6,10 +6,15 @@ import oracle
 from workloads import make_target_logits
 from workloads.gen import _rng
 
-# Attention tolerance.  Target: max |a-b| <= 1e-2 and, per (node, head) row,
-# max|a-b| / max|b| <= 1e-2.  The output is stored in bf16, whose rounding alone is up to
-# 2^-8 |b| (0.0156 at |b| = 4), so the absolute bound is scaled by max(1, row max |b|):
-# it is exactly 1e-2 wherever outputs stay below 1 in magnitude (all long-context rows).
+# Attention tolerance, against the fp64 oracle on the same bf16 inputs:
+#   max |a-b| <= 1e-2                                    (absolute, unscaled), and
+#   per (node, head) row  max|a-b| / max|b| <= 1e-2      ("row-relative": the row's largest
+#                                                         error over the row's largest magnitude)
+# An element-wise relative bound cannot hold for elements near zero with any bf16 output.
+# The output is stored in bf16: rounding alone costs up to half a unit in the last place,
+# 2^(floor(log2|b|) - 8), which is 0.0156 once |b| >= 4.  Outputs that large only occur in the
+# tiny-context edge cases (a handful of keys, no averaging); those tests, and only those, pass
+# `bf16_slack=True`, which adds exactly that half-ulp of the oracle value to the absolute bound.
 ATTN_MAX_ABS = 1e-2
 ATTN_ROW_REL = 1e-2
 ENTROPY_ABS = 1e-5
@@ -35,17 +40,39 @@ def widen(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
-def check_attention(got_bits: np.ndarray, want: np.ndarray):
-    """got: bf16 bits [nodes, Hq, d]; want: fp64 same shape."""
+def bf16_half_ulp(x: np.ndarray) -> np.ndarray:
+    """Half a unit in the last place of bf16 (8 significand bits) at magnitude |x|."""
+    mag = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(mag)) - 8.0)
+
+
+def check_attention(got_bits: np.ndarray, want: np.ndarray, bf16_slack: bool = False):
+    """got: bf16 bits [nodes, Hq, d]; want: fp64 same shape.  Returns (max abs error,
+    max row-relative error)."""
     got = widen(got_bits)
     assert np.isfinite(got).all()
     err = np.abs(got - want)
+    bound = ATTN_MAX_ABS + (bf16_half_ulp(want) if bf16_slack else 0.0)
+    worst = (err - bound).max()
+    assert worst <= 0.0, f"max abs err {err.max()} exceeds the bound by {worst}"
     row_mag = np.abs(want).max(axis=-1)
-    excess = err.max(axis=-1) / np.maximum(1.0, row_mag)
-    assert excess.max() <= ATTN_MAX_ABS, f"max abs err {err.max()} (scaled {excess.max()})"
     row_rel = err.max(axis=-1) / row_mag
     assert row_rel.max() <= ATTN_ROW_REL, f"max row-relative err {row_rel.max()}"
     return float(err.max()), float(row_rel.max())
+
+
+def check_logits(got, lg, k, ke):
+    """Outputs of sage_expand_topk (host arrays) against the oracle on the same logits."""
+    H, lse = oracle.softmax_entropy(lg)
+    idx = oracle.topk(lg, k)
+    Ht, alpha = oracle.confidence(lg, ke)
+    np.testing.assert_array_equal(got["topk_idx"], idx)
+    assert np.abs(got["entropy_full"] - H).max() <= ENTROPY_ABS
+    assert np.abs(got["entropy_topk"] - Ht).max() <= ENTROPY_ABS
+    assert np.abs(got["alpha"] - alpha).max() <= ENTROPY_ABS
+    assert np.abs(got["lse"] - lse).max() <= 1e-5 * max(1.0, np.abs(lse).max())
+    lp = oracle.topk_logprob(lg, idx, lse)
+    assert np.abs(got["topk_logprob"] - lp).max() <= 1e-5 * max(1.0, np.abs(lp).max())
 
 
 def oracle_attention_layer(c, layer):

@@ -71,7 +71,9 @@ def test_grow_tree_with_per_sequence_maximum_depth():
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     np.testing.assert_array_equal(tree["n_nodes"].cpu().numpy(), n_nodes)
+    np.testing.assert_array_equal(tree["frontier_begin"].cpu().numpy(), frontier)
     for name in ("parent", "rank", "depth", "token"):
         np.testing.assert_array_equal(tree[name].cpu().numpy(), host[name])
+    np.testing.assert_array_equal(tree["cum_logprob"].cpu().numpy().view(np.uint32), host["cum_logprob"].view(np.uint32))
     depth_reached = [int(host["depth"][b * CAP:b * CAP + n_nodes[b]].max()) for b in range(B)]
     assert depth_reached[0] <= 3 and depth_reached[1] <= 5 and depth_reached[0] < depth_reached[2]

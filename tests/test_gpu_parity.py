@@ -8,7 +8,7 @@ import torch
 
 import oracle
 import paper_2602_00523_b200 as sage
-from helpers import (ENTROPY_ABS, check_attention, dev_bf16, dev_f32, dev_i32, host_bits, oracle_attention_layer,
+from helpers import (ENTROPY_ABS, check_attention, check_logits, dev_bf16, dev_f32, dev_i32, host_bits, oracle_attention_layer,
                      oracle_logits_side, target_logits_for)
 from workloads import (TEMPLATES, bf16_bits, chain_tree, make_config, make_kv_cache, make_q, make_template,
                        random_tree, star_tree)
@@ -44,19 +44,6 @@ def gpu_logits(c, logits, k=None, ke=None, with_tree=True):
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     return {n: t.cpu().numpy() for n, t in o.items()}
-
-
-def check_logits(got, lg, k, ke):
-    H, lse = oracle.softmax_entropy(lg)
-    idx = oracle.topk(lg, k)
-    Ht, alpha = oracle.confidence(lg, ke)
-    np.testing.assert_array_equal(got["topk_idx"], idx)
-    assert np.abs(got["entropy_full"] - H).max() <= ENTROPY_ABS
-    assert np.abs(got["entropy_topk"] - Ht).max() <= ENTROPY_ABS
-    assert np.abs(got["alpha"] - alpha).max() <= ENTROPY_ABS
-    assert np.abs(got["lse"] - lse).max() <= 1e-5 * max(1.0, np.abs(lse).max())
-    lp = oracle.topk_logprob(lg, idx, lse)
-    assert np.abs(got["topk_logprob"] - lp).max() <= 1e-5 * max(1.0, np.abs(lp).max())
 
 
 # ------------------------------------------------------------------ ancestors
@@ -244,7 +231,9 @@ def test_tree_attention_edges(L, N, G):
     c = {"q": make_q(r, N, Hkv * G), **kv, "parent": tree["parent"], "node_offsets": np.array([0, N], np.int32),
          "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.11}
     got = gpu_attention(c)
-    check_attention(got[0], oracle_attention_layer(c, 0))
+    # tiny contexts: outputs of magnitude > 1, where the bf16 rounding of the output alone can
+    # exceed 1e-2; the bound gets the half-ulp of the oracle value added (here and nowhere else)
+    check_attention(got[0], oracle_attention_layer(c, 0), bf16_slack=True)
 
 
 def test_tree_attention_chain_and_star_trees():
@@ -276,6 +265,21 @@ def test_tree_attention_reports_bad_page_and_bad_tree():
     st = sage.new_status()
     gpu_attention(bad, status=st)
     assert int(st.item()) == sage.SAGE_STATUS_BAD_PAGE
+
+
+def test_tree_attention_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """Every on-device wait is bounded.  With the copy warp switched off nothing is ever in flight and
+    the first consumer wait can never be satisfied: the kernel must return, say SAGE_STATUS_TIMEOUT,
+    and an ordinary call right afterwards must still match the oracle."""
+    c = make_config(1)
+    st = sage.new_status()
+    sage.sage_debug_attention_waits(2_000_000, producer_off=True)        # about a millisecond per wait
+    try:
+        gpu_attention(c, status=st)
+    finally:
+        sage.sage_debug_attention_waits(0, producer_off=False)
+    assert int(st.item()) == sage.SAGE_STATUS_TIMEOUT
+    check_attention(gpu_attention(c)[0], oracle_attention_layer(c, 0))
 
 
 def test_tree_attention_is_deterministic():
@@ -367,6 +371,7 @@ def test_compact_kv_rejects_bad_path_without_touching_the_pool():
     assert st == sage.SAGE_STATUS_BAD_PATH
     np.testing.assert_array_equal(k2, kv["k_pool"])
     np.testing.assert_array_equal(v2, kv["v_pool"])
+    np.testing.assert_array_equal(sl, kv["seq_len"])          # a rejected sequence does not advance either
 
 
 # ------------------------------------------------------------------ whole round
@@ -392,7 +397,10 @@ def test_full_round_against_oracle(cfg):
     assert w_len.max() > 1                                    # the planted path was found
     out = gpu_attention(c)
     for layer in range(2):
-        check_attention(out[layer], oracle_attention_layer(c, layer))
+        # contexts cut to an eighth: outputs of magnitude > 2 occur, where the bf16 rounding of the
+        # output alone approaches 1e-2 (the full-size configurations are held to the plain bound in
+        # test_tree_attention_configs and in the configuration-4 / configuration-5 tests)
+        check_attention(out[layer], oracle_attention_layer(c, layer), bf16_slack=(cfg != 1))
     k2, v2, sl, st = run_compaction(c, g_path, g_len, 2)
     assert st == 0
     wk, wv, wl = oracle.compact_kv(c["k_pool"], c["v_pool"], c["page_table"], c["seq_len"], w_path, w_len, 64)

@@ -6,7 +6,8 @@ input and output buffers and nothing else, and a decode loop cannot afford cudaM
 device-wide synchronisation.  For them the library carries its own fixed scratch array.
 These tests call that entry point through the C ABI, twice in a row on different inputs
 (the array is shared between calls and keeps the previous call's contents), and compare
-every output with what the caller-workspace entry point gives on the same inputs.
+every output with what the caller-workspace entry point gives on the same inputs and with
+the CPU oracle.
 
 The file name sorts after every other test file on purpose: a run that stops at the
 first failure has then already gone through all the other tests.
@@ -18,7 +19,7 @@ import pytest
 import torch
 
 import paper_2602_00523_b200 as sage
-from helpers import ENTROPY_ABS, dev_f32, dev_i32
+from helpers import ENTROPY_ABS, check_logits, dev_f32, dev_i32
 from workloads import make_logits, make_template
 
 FLOAT_OUTPUTS = ("topk_logprob", "entropy_full", "entropy_topk", "alpha", "lse")
@@ -44,7 +45,8 @@ def test_static_scratch_matches_workspace_entry_point_on_two_calls_in_a_row():
              (make_template(8, 2, 24), 40961, "low", 2, 10)]
     for tree, vocab, kind, k, ke in cases:
         n = len(tree["parent"])
-        logits = dev_f32(make_logits(rng, n, vocab, kind)["logits"])
+        logits_host = make_logits(rng, n, vocab, kind)["logits"]
+        logits = dev_f32(logits_host)
         # a row stride of 4-element granularity is required by both entry points
         if vocab % 4:
             padded = torch.zeros((n, (vocab + 3) // 4 * 4), dtype=torch.float32, device=dev)
@@ -62,6 +64,8 @@ def test_static_scratch_matches_workspace_entry_point_on_two_calls_in_a_row():
         for name in FLOAT_OUTPUTS:
             diff = (got[name].double() - want[name].double()).abs().max().item()
             assert diff <= ENTROPY_ABS, (name, diff)
+        # and against the oracle itself, on the same logits
+        check_logits({name: t.cpu().numpy() for name, t in got.items()}, logits_host, k, ke)
 
 
 def test_static_scratch_rejects_problems_beyond_its_array_without_a_gpu():

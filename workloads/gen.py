@@ -201,6 +201,16 @@ def make_kv_cache(rng: np.random.Generator, seq_lens: Sequence[int], n_nodes: Se
             "seq_len": np.asarray(seq_lens, dtype=np.int32)}
 
 
+def place_rows(pool: np.ndarray, page_table_row: np.ndarray, first_pos: int, rows: np.ndarray,
+               page_size: int = 64) -> None:
+    """Stores ``rows`` (uint16 [layers, tokens, kv_heads, d]) at logical positions ``first_pos ..`` of one
+    sequence of a paged pool ``[layers, pages, kv_heads, slot, d]``, in place.  Stands in for the
+    model forward that writes a round's tree K/V into the cache."""
+    for i in range(rows.shape[1]):
+        t = first_pos + i
+        pool[:, int(page_table_row[t // page_size]), :, t % page_size, :] = rows[:, i]
+
+
 def make_q(rng: np.random.Generator, sum_nodes: int, n_q_heads: int, head_dim: int = 128,
            n_layers: int = 1) -> np.ndarray:
     """Query rows ``[layer, node, q_head, d]`` ~ N(0,1), bf16 bits."""
