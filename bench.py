@@ -438,10 +438,42 @@ def run_cuda(args):
         ms = max_over_ranks(ms, world, dev)
         return ms, attn_ms, clocks, seen
 
+    ws_cache = {"buf": ws_attn}
+
+    def ws_for(n_layers, n_nodes_cap):
+        """Attention workspace large enough for this shape (grown on demand, outside any timed region)."""
+        need = sage.sage_tree_attention_workspace_size(n_layers, 1, n_nodes_cap, HQ, HKV, D, used_pages)
+        if ws_cache["buf"].numel() < need:
+            ws_cache["buf"] = torch.empty(need, dtype=torch.uint8, device=dev)
+        return ws_cache["buf"]
+
+    def graph_time_us(fn, passes=3):
+        """GPU time of one call of fn(): its launches are captured in a CUDA graph once and replayed, so that
+        the host's per-call cost (Python, ctypes, tensor views) does not sit between the kernels."""
+        fn()                                          # first call outside the capture (per-device set-up, tensor maps)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(passes):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / passes
+
     def per_layer_attention_us(passes=3):
         """Attention launched layer by layer, as a model's forward does (other layers' work would sit
         in between): 80 single-layer calls walk over the 80 layers' K/V (5.5 GB), so no layer's K/V is
-        still in L2 when its turn comes.  Returns the mean microseconds per call (split-K + merge)."""
+        still in L2 when its turn comes.  Returns the mean GPU microseconds per call (attention + merge kernel;
+        the 80 calls are replayed as one CUDA graph)."""
         tree_parent = bank_parent[1, :N_NODES].contiguous()
         ws1 = torch.empty(max(16, sage.sage_tree_attention_workspace_size(1, 1, N_NODES, HQ, HKV, D, used_pages)),
                           dtype=torch.uint8, device=dev)
@@ -451,15 +483,7 @@ def run_cuda(args):
                 sage.sage_tree_attention(q_dev[layer:layer + 1], k_pool[layer:layer + 1], v_pool[layer:layer + 1],
                                          page_table, seq_len, tree_parent, node_offsets, 1.0 / np.sqrt(D),
                                          out=attn_out[layer:layer + 1], ws=ws1, status=status)
-        sweep()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(passes):
-            sweep()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)
+        return graph_time_us(sweep, passes) / N_LAYERS
 
     def attention_by_tree_size(reps=5):
         """The 80-layer attention launch alone for trees of 16 ... 60 nodes at the same 16k context
@@ -473,8 +497,9 @@ def run_cuda(args):
             offs = torch.tensor([0, n], dtype=torch.int32, device=dev)
             qn = q_dev[:, :n].contiguous()
             on = torch.empty_like(qn)
+            wsn = ws_for(N_LAYERS, n)
             call = lambda: sage.sage_tree_attention(qn, k_pool, v_pool, page_table, seq_len, tp, offs, 1.0 / np.sqrt(D),
-                                                    out=on, ws=ws_attn, status=status)
+                                                    out=on, ws=wsn, status=status)
             call(); call()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
@@ -494,7 +519,8 @@ def run_cuda(args):
     def attention_latency(passes=2):
         """Single-layer calls in the latency regime (draft-side attention, level-by-level growth, plain
         decode): contexts of 2048 and 16384 tokens, trees of 1 / 10 / 60 nodes.  Each pass walks over all
-        layers' K/V, so no call finds its K/V in L2.  Microseconds per call, launch gaps included."""
+        layers' K/V, so no call finds its K/V in L2.  GPU microseconds per call (CUDA-graph replay of the 80
+        calls: kernel time and the gaps between kernels, without the host's per-call cost)."""
         from workloads import chain_tree, make_template as mk
         rows = []
         for ctx in (2048, 16384):
@@ -504,27 +530,67 @@ def run_cuda(args):
                 offs = torch.tensor([0, n], dtype=torch.int32, device=dev)
                 qs = [q_dev[layer:layer + 1, :n].contiguous() for layer in range(N_LAYERS)]
                 on = torch.empty_like(qs[0])
+                wsn = ws_for(1, n)
 
                 def sweep():
                     for layer in range(N_LAYERS):
                         sage.sage_tree_attention(qs[layer], k_pool[layer:layer + 1], v_pool[layer:layer + 1], page_table, sl,
-                                                 tp, offs, 1.0 / np.sqrt(D), out=on, ws=ws_attn, status=status)
-                sweep()
-                torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                for _ in range(passes):
-                    sweep()
-                e1.record()
-                torch.cuda.synchronize()
-                rows.append({"context": ctx, "nodes": n, "us_per_call": e0.elapsed_time(e1) * 1e3 / (passes * N_LAYERS)})
+                                                 tp, offs, 1.0 / np.sqrt(D), out=on, ws=wsn, status=status)
+                rows.append({"context": ctx, "nodes": n, "us_per_call": graph_time_us(sweep, passes) / N_LAYERS})
         return rows
+
+    def policy_comparison(rounds=12, p_acc=0.8, gamma=0.9):
+        """Algorithm 1 as a device-side loop (no host round trip between rounds) under a synthetic acceptance
+        process (level l of the greedy path agrees with probability p * gamma^(l-1); lower-ranked candidates
+        geometrically less often), for four tree policies on this workload's shapes: SD-Chain, a static
+        SD-Tree, entropy-selected templates (look-ahead) and trees grown level by level with the depth
+        steered by the acceptance history.  Rounds/s and accepted tokens/s; the stand-in target's few
+        torch indexing kernels per round are inside the timing."""
+        from paper_2602_00523_b200.decode_loop import DecodeLoop, SyntheticTarget
+        from workloads import TEMPLATES, acceptance_picks, chain_tree, make_loop_logits
+        cap = sage.SAGE_MAX_NODES
+        grow = cap + (rounds + 3) * MAX_PATH
+        pages_loop = (L_PREFIX + grow + P - 1) // P
+        assert pages_loop <= n_pages
+        pt_loop = torch.from_numpy(_rng(CFG, 1).permutation(n_pages)[:pages_loop].astype(np.int32)).to(dev).view(1, -1)
+        rr = _rng(CFG, 700)
+        # draft distributions with a clear first choice and plausible alternatives, sharper or flatter per round
+        draft = [torch.from_numpy(make_loop_logits(rr, cap, V, kd)).to(dev) for kd in ("steps:9.5", "low", "steps:8", "steps:10.5")]
+        picks = acceptance_picks(rr, 64, cap, 8, K_TOP, p_acc, gamma)
+        noise = torch.empty((cap, V), dtype=torch.float32, device=dev).normal_(generator=gen)
+        q64 = torch.empty((N_LAYERS, cap, HQ, D), dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+        specs = [("sd_chain_depth8", "chain", dict(trees=[chain_tree(9)])),
+                 ("sd_tree_static_4x6", "static", dict(trees=[make_template(4, 6, N_NODES)])),
+                 ("sage_templates", "templates", dict(trees=[make_template(d_, w_, N_NODES) for d_, w_, _ in TEMPLATES],
+                                                      thresholds=[0.8, 0.4, 0.1])),
+                 ("sage_dynamic_history", "dynamic", dict())]
+        rows = []
+        for name, pol, kw in specs:
+            loop = DecodeLoop(policy=pol, draft_logits=draft, target=SyntheticTarget(noise, picks, K_TOP), k=K_TOP,
+                              k_entropy=K_ENT, q=q64, k_pool=k_pool, v_pool=v_pool, page_table=pt_loop, prefix_len=L_PREFIX,
+                              max_path=MAX_PATH, n_budget=N_NODES, rounds_capacity=rounds + 3, **kw)
+            loop.run(3)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            loop.run(rounds)
+            e1.record()
+            torch.cuda.synchronize()
+            if int(loop.status.item()) != 0:
+                raise RuntimeError("device status in the policy loop: " + sage.status_string(int(loop.status.item())))
+            t_ms = e0.elapsed_time(e1)
+            plen = loop.rec["path_len"][3:3 + rounds].float()
+            rows.append({"policy": name, "rounds_per_s": rounds / (t_ms * 1e-3), "accepted_tokens_per_s": float(plen.sum()) / (t_ms * 1e-3),
+                         "mean_tokens_per_round": float(plen.mean()), "mean_tree_nodes": float(loop.rec["n_nodes"][3:3 + rounds].float().mean()),
+                         "rounds": rounds})
+        return {"acceptance_process": {"p": p_acc, "gamma": gamma}, "node_budget": N_NODES, "layers": N_LAYERS, "results": rows}
 
     ms, attn_ms, clocks, _ = timed(False)
     other_us = {k: (float(np.mean([a.elapsed_time(b) for a, b in v])) * 1e3 if v else None) for k, v in other_events.items()}
     layer_us = None if args.no_per_layer else per_layer_attention_us()
     by_tree = None if args.no_sweeps else attention_by_tree_size()
     latency = None if args.no_sweeps else attention_latency()
+    policies = None if args.no_policies else policy_comparison()
     if int(status.item()) != 0:
         raise RuntimeError("device status: " + sage.status_string(int(status.item())))
     e2e_ms, _, _, seen = timed(True)
@@ -602,6 +668,7 @@ def run_cuda(args):
             "roofline_hbm_bound": hbm_entry,
             "attention_by_tree_size": by_tree,
             "attention_latency": latency,
+            "policies": policies,
             "other_launches": {
                 "expand_topk_draft_k10": None if not other_us["expand_draft"] else {
                     "us": other_us["expand_draft"], "gbs": logits_bytes / (other_us["expand_draft"] * 1e-6) / 1e9,
@@ -617,8 +684,8 @@ def run_cuda(args):
             "attention_per_layer": None if layer_us is None else {
                 "us_per_call": layer_us, "tflops": flops / N_LAYERS / (layer_us * 1e-6) / 1e12,
                 "gbs": kv_bytes / N_LAYERS / (layer_us * 1e-6) / 1e9,
-                "note": "80 single-layer calls walking over all layers' K/V (attention + merge kernels, launch "
-                        "gaps included)"},
+                "note": "80 single-layer calls walking over all layers' K/V (attention + merge kernels), replayed as "
+                        "one CUDA graph"},
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
@@ -639,6 +706,8 @@ def main():
                     help="skip the layer-by-layer attention timing (profiler launch lists of the round alone)")
     ap.add_argument("--no-sweeps", action="store_true",
                     help="skip the tree-size sweep and the latency sweep of the attention call")
+    ap.add_argument("--no-policies", action="store_true",
+                    help="skip the device-side decode loop under the four tree policies")
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip timing the CPU oracle (profiler captures)")
     args = ap.parse_args()

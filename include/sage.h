@@ -255,6 +255,13 @@ const char *sage_status_string(int code);
  * to run the time-out path without faulting or hanging the device; leave it alone otherwise. */
 void sage_debug_attention_waits(long long wait_cycles, int producer_off);
 
+/* sage_tree_attention has two schedules and picks one per launch: a streaming one (one resident thread
+ * block per multiprocessor walks an equal share of all the work) for long, HBM-bound launches, and a
+ * split one (a grid over context slices, row pairs and KV heads, plus a merge) for tensor-bound trees
+ * and short launches.  schedule = 1 forces the streaming one, 2 the split one, anything else restores
+ * the automatic choice.  For tests and measurements (no counterpart in the paper). */
+void sage_debug_attention_schedule(int schedule);
+
 #ifdef __cplusplus
 }
 #endif

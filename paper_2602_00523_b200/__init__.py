@@ -16,7 +16,7 @@ _BINDING_NAMES = (
     "sage_expand_topk", "sage_expand_topk_workspace_size", "sage_expand_topk_static", "sage_select_tree",
     "sage_build_ancestor_mask", "sage_grow_tree", "sage_update_history", "make_history_policy",
     "SageHistoryPolicy", "sage_tree_attention", "sage_tree_attention_workspace_size",
-    "sage_accept", "sage_compact_kv", "sage_debug_attention_waits",
+    "sage_accept", "sage_compact_kv", "sage_debug_attention_waits", "sage_debug_attention_schedule",
     "SAGE_OK", "SAGE_ERR_INVALID_ARG", "SAGE_ERR_UNSUPPORTED", "SAGE_ERR_WORKSPACE", "SAGE_ERR_CUDA",
     "SAGE_ERR_TOO_LARGE", "SAGE_STATIC_SCRATCH_BYTES",
     "SAGE_STATUS_BAD_TREE", "SAGE_STATUS_BAD_PAGE", "SAGE_STATUS_TIMEOUT", "SAGE_STATUS_BAD_PATH",

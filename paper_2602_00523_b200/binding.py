@@ -90,6 +90,8 @@ _lib.sage_compact_kv.restype = _i
 _lib.sage_compact_kv.argtypes = [_vp, _vp, _i64, _i, _i, _vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.sage_debug_attention_waits.restype = None
 _lib.sage_debug_attention_waits.argtypes = [ctypes.c_longlong, _i]
+_lib.sage_debug_attention_schedule.restype = None
+_lib.sage_debug_attention_schedule.argtypes = [_i]
 _lib.sage_status_string.restype = ctypes.c_char_p
 _lib.sage_status_string.argtypes = [_i]
 
@@ -289,6 +291,11 @@ def sage_debug_attention_waits(wait_cycles: int = 0, producer_off: bool = False)
     """Cycle budget of the attention kernel's on-device waits (0 = default) and, for tests of the
     time-out path, a switch that keeps its copy warp from issuing anything."""
     _lib.sage_debug_attention_waits(int(wait_cycles), 1 if producer_off else 0)
+
+
+def sage_debug_attention_schedule(schedule: int = 0) -> None:
+    """0: the library picks the attention schedule per launch; 1: streaming; 2: split."""
+    _lib.sage_debug_attention_schedule(int(schedule))
 
 
 def sage_accept(parent, draft_token, target_argmax, node_offsets, max_path: int, *, out=None, status=None, stream=None):

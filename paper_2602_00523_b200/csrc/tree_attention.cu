@@ -1043,6 +1043,30 @@ static int row_pairs(int sum_nodes, int G) {
 
 static long long g_wait_cycles = kWaitCyclesDefault;
 static int g_producer_off = 0;
+static int g_schedule = 0;     // 0: chosen per launch, 1: streaming, 2: split
+
+// The split schedule (tree_attention_split.cu).
+namespace split {
+size_t workspace_size(int n_layers, int batch, int sum_nodes, int n_q_heads, int n_kv_heads, int max_pages_per_seq);
+int launch(const void* q, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+           const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
+           int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
+           int producer_off, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream);
+}  // namespace split
+
+// Which schedule runs a launch.  The streaming schedule (this file) wins where the work is HBM-bound and
+// long: trees of up to 256 query rows per KV head (one thread block per gang, nothing idles) with at least
+// `kStreamMinSteps` 128-key steps for every SM.  Tensor-bound trees (a gang's second block would mostly
+// repeat the first one's waits) and short launches (single layers, short contexts: fixed costs dominate)
+// go to the split schedule.
+constexpr int kStreamMinSteps = 16;
+static bool use_streaming(int n_layers, int batch, int sum_nodes, int n_kv_heads, int G, int max_pages_per_seq) {
+    if (g_schedule == 1) return true;
+    if (g_schedule == 2) return false;
+    if (row_pairs(sum_nodes, G) > 1) return false;
+    const long long steps = (long long)n_layers * batch * n_kv_heads * ((max_pages_per_seq + 1) / 2);   // upper bound
+    return steps >= (long long)kStreamMinSteps * resident_ctas();
+}
 
 }  // namespace sage
 
@@ -1054,14 +1078,19 @@ extern "C" size_t sage_tree_attention_workspace_size(int n_layers, int batch, in
         n_q_heads % n_kv_heads)
         return 0;
     (void)head_dim;
-    // two partial slots (head and tail of its range) per resident CTA, independent of the problem size
-    return (size_t)resident_ctas() * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float);
+    // streaming schedule: two partial slots (head and tail of its range) per resident CTA, independent of the
+    // problem size; split schedule: one partial per context slice.  Either may run, so the larger is asked for.
+    const size_t streaming = (size_t)resident_ctas() * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float);
+    const size_t split_ws = split::workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads, max_pages_per_seq);
+    return streaming > split_ws ? streaming : split_ws;
 }
 
 extern "C" void sage_debug_attention_waits(long long wait_cycles, int producer_off) {
     g_wait_cycles = wait_cycles > 0 ? wait_cycles : kWaitCyclesDefault;
     g_producer_off = producer_off ? 1 : 0;
 }
+
+extern "C" void sage_debug_attention_schedule(int schedule) { g_schedule = (schedule == 1 || schedule == 2) ? schedule : 0; }
 
 extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void* v_pool, int64_t layer_stride_elems,
                                    int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
@@ -1087,6 +1116,18 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     const size_t need = sage_tree_attention_workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads,
                                                            head_dim, max_pages_per_seq);
     if (!ws || ws_bytes < need || ((uintptr_t)ws & 15)) return SAGE_ERR_WORKSPACE;
+    if ((long long)n_layers * batch * n_kv_heads > 65535 &&
+        !use_streaming(n_layers, batch, sum_nodes, n_kv_heads, G, max_pages_per_seq))
+        return SAGE_ERR_UNSUPPORTED;                    // grid limit of the split schedule
+    if (!use_streaming(n_layers, batch, sum_nodes, n_kv_heads, G, max_pages_per_seq)) {
+        CUtensorMap kmap, vmap;
+        if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
+            !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
+            return SAGE_ERR_CUDA;
+        return split::launch(q, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent, node_offsets, batch,
+                             sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status, g_wait_cycles, g_producer_off,
+                             kmap, vmap, as_stream(stream));
+    }
     const int n_ctas = resident_ctas();
     AttnParams p{};
     p.n_rp = row_pairs(sum_nodes, G);

@@ -43,12 +43,15 @@ def _build():
                 seq_len=dev_i32([L]), parent=dev_i32(tree["parent"]), offs=dev_i32([0, N]))
 
 
-def test_attention_80_layers_sampled_layers_match_the_oracle_and_all_outputs_are_finite():
+@pytest.mark.parametrize("schedule", [0, 1], ids=["as_benchmarked", "streaming"])
+def test_attention_80_layers_sampled_layers_match_the_oracle_and_all_outputs_are_finite(schedule):
     w = _build()
+    sage.sage_debug_attention_schedule(schedule)
     st = sage.new_status()
     out = sage.sage_tree_attention(w["q"], w["k"], w["v"], w["page_table"], w["seq_len"], w["parent"], w["offs"],
                                    1.0 / np.sqrt(D), status=st)
     torch.cuda.synchronize()
+    sage.sage_debug_attention_schedule(0)
     assert int(st.item()) == 0, sage.status_string(int(st.item()))
     assert bool(torch.isfinite(out.float()).all())
     offs = np.array([0, N], np.int32)

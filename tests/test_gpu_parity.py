@@ -199,14 +199,22 @@ def test_select_tree_edges_and_handover():
 
 
 # ------------------------------------------------------------------ attention
+@pytest.fixture(params=[1, 2], ids=["streaming", "split"])
+def schedule(request):
+    """sage_tree_attention picks one of its two schedules per launch; the parity tests force each in turn."""
+    sage.sage_debug_attention_schedule(request.param)
+    yield request.param
+    sage.sage_debug_attention_schedule(0)
+
+
 @pytest.mark.parametrize("cfg", [1, 2, 3])
-def test_tree_attention_configs(cfg):
+def test_tree_attention_configs(cfg, schedule):
     c = make_config(cfg)
     got = gpu_attention(c)
     check_attention(got[0], oracle_attention_layer(c, 0))
 
 
-def test_tree_attention_config4_three_layers_full_context():
+def test_tree_attention_config4_three_layers_full_context(schedule):
     c = make_config(4, n_layers=3)                           # L = 16384, shuffled pages, 60 nodes
     got = gpu_attention(c)                                   # stacked-layer launch
     for layer in range(3):
@@ -215,7 +223,7 @@ def test_tree_attention_config4_three_layers_full_context():
     check_attention(one[0], oracle_attention_layer(c, 1))
 
 
-def test_tree_attention_config5_ragged_batch():
+def test_tree_attention_config5_ragged_batch(schedule):
     c = make_config(5)
     got = gpu_attention(c)
     check_attention(got[0], oracle_attention_layer(c, 0))
@@ -223,7 +231,7 @@ def test_tree_attention_config5_ragged_batch():
 
 @pytest.mark.parametrize("L,N,G", [(0, 1, 8), (0, 64, 8), (1, 7, 4), (63, 2, 8), (64, 64, 8), (65, 33, 2),
                                    (127, 60, 8), (200, 64, 1), (1000, 17, 8), (4097, 64, 8)])
-def test_tree_attention_edges(L, N, G):
+def test_tree_attention_edges(L, N, G, schedule):
     r = rng(L * 100 + N)
     Hkv = 2
     tree = random_tree(r, N)
@@ -236,7 +244,7 @@ def test_tree_attention_edges(L, N, G):
     check_attention(got[0], oracle_attention_layer(c, 0), bf16_slack=True)
 
 
-def test_tree_attention_chain_and_star_trees():
+def test_tree_attention_chain_and_star_trees(schedule):
     r = rng(9)
     for tree in (chain_tree(40), star_tree(50)):
         N = len(tree["parent"])
@@ -246,7 +254,7 @@ def test_tree_attention_chain_and_star_trees():
         check_attention(gpu_attention(c)[0], oracle_attention_layer(c, 0))
 
 
-def test_tree_attention_reports_bad_page_and_bad_tree():
+def test_tree_attention_reports_bad_page_and_bad_tree(schedule):
     c = make_config(1)
     bad = dict(c)
     bad["page_table"] = c["page_table"].copy()
@@ -267,7 +275,7 @@ def test_tree_attention_reports_bad_page_and_bad_tree():
     assert int(st.item()) == sage.SAGE_STATUS_BAD_PAGE
 
 
-def test_tree_attention_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+def test_tree_attention_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable(schedule):
     """Every on-device wait is bounded.  With the copy warp switched off nothing is ever in flight and
     the first consumer wait can never be satisfied: the kernel must return, say SAGE_STATUS_TIMEOUT,
     and an ordinary call right afterwards must still match the oracle."""
@@ -282,7 +290,7 @@ def test_tree_attention_wait_that_runs_out_reports_timeout_and_leaves_the_contex
     check_attention(gpu_attention(c)[0], oracle_attention_layer(c, 0))
 
 
-def test_tree_attention_is_deterministic():
+def test_tree_attention_is_deterministic(schedule):
     c = make_config(3, scale_down=4)
     np.testing.assert_array_equal(gpu_attention(c), gpu_attention(c))
 

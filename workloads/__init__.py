@@ -10,4 +10,5 @@ from .gen import (  # noqa: F401
     bf16_bits, bf16_to_f32, make_template, random_tree, chain_tree, star_tree,
     make_kv_cache, make_q, place_rows, make_logits, make_target_logits, make_config,
     markov_entropy_states, TEMPLATES, CONFIG_NAMES, seed_for,
+    acceptance_picks, make_loop_logits, NO_CANDIDATE,
 )

@@ -230,6 +230,8 @@ def make_logits(rng: np.random.Generator, rows: int, vocab: int, kind) -> Dict[s
       "mixed" N(0,1) * s, s drawn from {0.5, 2, 8}, plus a planted peak
               = row max + U[0.5,4] at a random index
       "mid:<m>" N(0,1) plus a planted peak = row max + m           (tunable)
+      "steps:<m>" N(0,1) plus eight planted peaks at row max + m, m - 1, m - 2, ...
+              (a draft that has a clear first choice and plausible alternatives)
     """
     kinds = [kind] * rows if isinstance(kind, str) else list(kind)
     out = np.empty((rows, vocab), dtype=np.float32)
@@ -241,7 +243,14 @@ def make_logits(rng: np.random.Generator, rows: int, vocab: int, kind) -> Dict[s
             x *= np.float32(0.5)
         elif kd == "mixed":
             x *= np.float32([0.5, 2.0, 8.0][int(rng.integers(0, 3))])
-        if kd != "high":
+        if kd.startswith("steps:"):
+            top = float(kd[6:])
+            base = x.max()
+            idx = rng.choice(vocab, size=8, replace=False)
+            for j, ix in enumerate(idx):
+                x[int(ix)] = np.float32(base + np.float32(top - j))
+            peak[r] = int(idx[0])
+        elif kd != "high":
             if kd == "low":
                 margin = rng.uniform(6.0, 10.0)
             elif kd == "mixed":
@@ -291,6 +300,41 @@ def markov_entropy_states(rng: np.random.Generator, rounds: int, p_stay: float =
         if rng.random() >= p_stay:
             s = 1 - s
     return out
+
+
+# --------------------------------------------------------------------------
+# Synthetic acceptance process for multi-round decode loops.  The target model
+# is replaced by a table of draws: for a node whose children sit at level l,
+# the target's greedy token equals the draft's rank-R candidate with
+# P(R = r) = p_l (1 - p_l)^r,  p_l = p * gamma^(l-1)   (r < k), and no candidate
+# otherwise.  With a chain (only rank-0 children) level l is then accepted with
+# probability p * gamma^(l-1), the process of the paper's expected-acceptance
+# theorem (Section 4.2).  The table is data: both the CPU oracle loop and the
+# device loop look the draws up, neither draws anything itself.
+# --------------------------------------------------------------------------
+NO_CANDIDATE = 255
+
+
+def acceptance_picks(rng: np.random.Generator, rounds: int, n_slots: int, max_level: int, k: int,
+                     p: float, gamma: float) -> np.ndarray:
+    """uint8 [rounds, n_slots, max_level + 1]: entry [r, u, l] is the candidate rank the target agrees
+    with at node slot u in round r if u's children are at level l (l >= 1; column 0 is unused), or
+    NO_CANDIDATE."""
+    out = np.full((rounds, n_slots, max_level + 1), NO_CANDIDATE, dtype=np.uint8)
+    for lvl in range(1, max_level + 1):
+        pl = float(p) * float(gamma) ** (lvl - 1)
+        # number of failures before the first success of a Bernoulli(pl) sequence
+        draws = rng.geometric(pl, size=(rounds, n_slots)) - 1 if pl > 0 else np.full((rounds, n_slots), k)
+        out[:, :, lvl] = np.where(draws < k, draws, NO_CANDIDATE).astype(np.uint8)
+    return out
+
+
+def make_loop_logits(rng: np.random.Generator, rows: int, vocab: int, kind: str) -> np.ndarray:
+    """Draft logits rows for the decode loops: as make_logits, with token 0 pushed far down so that it is
+    never among a row's top candidates (the loops use it as the token that matches no draft node)."""
+    lg = make_logits(rng, rows, vocab, kind)["logits"]
+    lg[:, 0] = np.float32(-30.0)
+    return lg
 
 
 # --------------------------------------------------------------------------
