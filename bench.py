@@ -43,10 +43,12 @@ WORKLOAD = "config4: qwen2.5-vl-72b layer shape 64/8/128 bf16, 16384-token prefi
            "page 64 shuffled, 60-node tree, 80 layers, logits 60x152064 fp32"
 
 
-# DRAM bytes per layer of the attention launch as counted by ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of a 9-layer capture / 9; traffic grows in proportion to the layer count:
-# every layer streams its own K/V once).  None = the kernel changed since the counters were taken.
-ATTN_DRAM_BYTES_PER_LAYER = None
+# DRAM bytes per layer of the benchmark's attention launch (split schedule, 60-node tree) as counted by
+# ncu: dram__bytes_read.sum + dram__bytes_write.sum = 615.30 MB + 3.81 MB over 9 layers
+# (profiles/tree_attention_split_kernel_config4_9layers.md).  Traffic grows in proportion to the layer
+# count: every layer streams its own K/V once.  Set to None whenever that kernel changes until the
+# counters are taken again.
+ATTN_DRAM_BYTES_PER_LAYER = 619.11e6 / 9
 
 
 def load_peaks():
@@ -619,7 +621,9 @@ def run_cuda(args):
                             "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
                                       f"rows), attention, acceptance and compaction of 1 of the {N_LAYERS} layers; "
                                       "the other layers are extrapolated"}
-        launches = 3 + 2 + 2 + 2 + 1 + 2      # expand (3), select + hand-over, attention + merge, target top-1 (2), accept, compact (2)
+        # expand (3), select + hand-over (2), attention (1: at this shape the split schedule runs with one context
+        # slice per CTA, so no merge kernel is launched), target top-1 (2), accept (1), compact + advance (2)
+        launches = 3 + 2 + 1 + 2 + 1 + 2
         # Which tensor peak applies: the burst figure when the SM clock stayed at its maximum through the
         # timed region, the sustained one when the power cap pulled it down.  Both fractions are printed.
         sm, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")

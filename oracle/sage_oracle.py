@@ -160,7 +160,9 @@ def confidence(logits: np.ndarray, k_entropy: int):
 # paper leaves the mapping from the real-valued (D, W) to a concrete tree
 # open; here a tree template is picked by comparing alpha with descending
 # thresholds.  The comparison is done on the fp32 alpha it is handed, in
-# fp32, exactly as the library does.
+# fp32: alpha arrives as an fp32 array (the storage type of the confidence
+# outputs), and comparing it in any wider type against thresholds that are
+# themselves fp32 policy constants would decide a different question.
 # --------------------------------------------------------------------------
 def select_tree(alpha, thresholds, d_min=3.0, d_max=8.0, w_min=2.0, w_max=10.0):
     """Returns (template_id int32 [B], D_cont fp64 [B], W_cont fp64 [B]).
@@ -280,7 +282,9 @@ def compact_kv(k_pool, v_pool, page_table, seq_len, path, path_len, page_size):
 # rule is invented); a level l exists iff l <= D(alpha); nodes are added in
 # breadth-first order (parents by index, ranks ascending) until N_max nodes.
 # Decisions are taken in fp64 on the fp32 inputs; cumulative log-probabilities
-# are fp32 sums (the library does the same).  "parity unpinned" for these
+# are fp32 sums, because fp32 is the storage type of the log-probabilities the
+# caller hands over and of the per-node array the sums are kept in from one
+# level to the next.  "parity unpinned" for these
 # readings; the level-wise construction itself is pinned against the path rule
 # evaluated directly on every path of a full k-ary tree.
 # --------------------------------------------------------------------------
