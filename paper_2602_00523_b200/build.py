@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsage.so")
-SOURCES = ["tree_ops.cu", "logits_stats.cu", "tree_attention.cu", "tree_attention_split.cu"]
+SOURCES = ["tree_ops.cu", "logits_stats.cu", "tree_attention.cu", "tree_attention_rows.cu", "tree_attention_split.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -35,14 +35,25 @@
 namespace sage {
 
 constexpr int kRowTile = 128;                  // query rows per MMA tile
-constexpr int kRowsPerCta = 2 * kRowTile;
+constexpr int kRowsPerCta = kRowTile;          // one row tile per CTA; its steps alternate between two slots
 constexpr int kStepKeys = 2 * kPageSize;       // keys per pipeline step
-constexpr int kKStages = 3;                    // K tiles in flight
-constexpr int kVStages = 2;                    // V tiles in flight
-constexpr int kRing = 4;                       // barrier pairs of the copy ring (ring steps in flight <= 2)
 constexpr int kPageHalfBytes = kPageSize * 64 * 2;          // one TMA box: 64 keys x 64-wide d-half = 8 KB
 constexpr int kTileHalfBytes = kStepKeys * 64 * 2;          // one d-half of a 128-key tile: 16 KB
 constexpr int kTileBytes = 2 * kTileHalfBytes;              // K or V tile of one step: 32 KB
+constexpr int kMaxRing = 8;
+// The kernel comes in two forms.  Single: one CTA holds the whole K and V tile of a step.  Pair: two
+// CTAs of a cluster (the two SMs of a TPC) work on two row tiles with one MMA stream (cta_group::2, M = 256);
+// each holds half of every K tile (64 of the 128 keys) and half of every V tile (64 of the 128 head
+// dimensions), so a step's K and V enter the pair's shared memory once.
+template <bool kPair>
+struct Cfg {
+    static constexpr int kStages = kPair ? 6 : 3;                       // K tiles, and V tiles, in flight per CTA
+    static constexpr int kDepth = kStages;                              // ring steps the copies run ahead of the MMAs
+    static constexpr int kRing = kStages + 1;                           // barrier pairs of the copy ring (> kDepth)
+    static constexpr int kTile = kPair ? kTileBytes / 2 : kTileBytes;   // this CTA's part of a step's K (or V) tile
+    static constexpr int kKHalf = kTile / 2;                            // distance between the two d-halves of its K part
+    static_assert(kRing <= kMaxRing, "ring barriers");
+};
 constexpr int kQTileBytes = kRowTile * kHeadDim * 2;        // 32 KB
 constexpr int kQHalfBytes = kRowTile * 64 * 2;              // one 64-wide d-half of a Q tile: 16 KB
 constexpr int kAttnThreads = 384;              // 2 softmax warpgroups + one warpgroup of TMA warp, MMA warp and two idle warps
@@ -51,8 +62,8 @@ constexpr long long kWaitCyclesDefault = 4000000000ll;   // ~2 s at 2 GHz: far b
 
 struct AttnParams {
     __nv_bfloat16* out;
-    float* part_o;     // [gang][2][gang member][256 rows][128]   unnormalised
-    float* part_ml;    // [gang][2][gang member][256 rows][2]     (reference max in log2 units, l)
+    float* part_o;     // [gang][2][gang member][128 rows][128]   unnormalised
+    float* part_ml;    // [gang][2][gang member][128 rows][2]     (reference max in log2 units, l)
     const int32_t* page_table;
     const int32_t* seq_len;
     const int32_t* parent;
@@ -60,28 +71,33 @@ struct AttnParams {
     int32_t* status;
     int n_layers, batch, sum_nodes, n_pages, max_pages;
     int Hq, Hkv, G;
-    int n_gangs, n_rp;         // gangs in the launch, CTAs per gang (row pairs of the largest possible tree)
+    int n_gangs, n_rp;         // gangs in the launch, CTAs per gang (row tiles of the largest possible tree)
     float scale_log2;          // sm_scale * log2(e)
     long long wait_cycles;     // budget of every on-device wait
     int producer_off;          // diagnostics: the TMA warp issues no copies (every consumer wait then runs out)
 };
 
 struct __align__(16) Shared {
-    uint64_t kv_full[kRing];   // ring step r: the K tile of its step and the V tile of the step before have landed
-    uint64_t kv_done[kRing];   // ring step r: every MMA that reads those tiles has finished
-    uint64_t s_full[2];        // [row tile]: scores of a step are in TMEM
-    uint64_t p_full[2];        // [row tile]: probabilities of a step are in TMEM
-    uint64_t o_full[2];        // [row tile]: every MMA of the segment has finished
-    uint64_t q_free;           // the segment's last score MMAs have read the query tiles
-    uint64_t q_ready;          // the query tiles of the segment are in shared memory
+    uint64_t kv_full[kMaxRing];    // ring step r: the K tile of its step and the V tile of two steps back have landed
+    uint64_t kv_done[kMaxRing];    // ring step r: every MMA that reads those tiles has finished
+    uint64_t s_full[2];        // [slot]: scores of a step are in TMEM
+    uint64_t p_full[2];        // [slot]: probabilities of a step are in TMEM
+    uint64_t o_full[2];        // [slot]: every MMA of the slot's part of the segment has finished
+    uint64_t epi_done;         // the softmax warps have read both accumulators of the segment
+    uint64_t q_free;           // the segment's last score MMAs have read the query tile
+    uint64_t q_ready;          // the query tile of the segment is in shared memory
     uint64_t drain;            // abort path: everything issued so far has retired
+    volatile uint32_t eflag[2][4];     // [slot][quadrant]: segment number whose (reference, sum) this warp has posted
     long long range_begin, range_end;
     int first_lg, first_b, first_s0;
     uint32_t tmem_base;
+    uint32_t peer_abort;       // pair form: cluster address of the other CTA's abort flag (0: none)
     volatile int abort;
 };
-constexpr int kSmemBytes = 1024 /*align*/ + 2 * kQTileBytes + (kKStages + kVStages) * kTileBytes + (int)sizeof(Shared);
+// the same for both forms: a query tile and 6 x 32 KB (or 12 x 16 KB) of K and V
+constexpr int kSmemBytes = 1024 /*align*/ + kQTileBytes + 6 * kTileBytes + (int)sizeof(Shared);
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
+static_assert(2 * Cfg<false>::kStages * Cfg<false>::kTile == 6 * kTileBytes && 2 * Cfg<true>::kStages * Cfg<true>::kTile == 6 * kTileBytes, "ring size");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -95,22 +111,43 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// kCluster: the barrier also takes arrivals from the other CTA of the pair
+template <bool kCluster = false>
 __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    if (kCluster)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_addr(const volatile void* ptr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(const_cast<const void*>(ptr))), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// The CTA (and, in the pair form, its partner) stops: every wait returns false from here on.
+__device__ __forceinline__ void raise_abort(Shared* sh) {
+    sh->abort = 1;
+    if (sh->peer_abort) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(sh->peer_abort), "r"(1) : "memory");
+}
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+template <bool kCluster = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, const AttnParams& p) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try<kCluster>(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 64; ++i)
-            if (mbar_try(bar, parity)) return true;
+            if (mbar_try<kCluster>(bar, parity)) return true;
         if (sh->abort) return false;
         if (clock64() - t0 > p.wait_cycles) {
-            sh->abort = 1;
+            raise_abort(sh);
             report_status(p.status, SAGE_STATUS_TIMEOUT);
             return false;
         }
@@ -139,17 +176,19 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
 // ---- tcgen05 --------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// One lane of a converged warp; the same lane every time for a full mask.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t e;
-    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
-    return e != 0;
-}
-// The helpers below are called by a whole converged warp so that their operands stay warp-uniform;
-// only the `leader` lane executes the instruction.
-__device__ __forceinline__ void tc_commit(bool leader, uint64_t* bar) {
-    if (leader)
+// Issued by the one thread that issues the MMAs.
+// Pair form: the arrival goes to the barrier at this offset in both CTAs, or (`both` false) in this one only.
+template <bool kPair>
+__device__ __forceinline__ void tc_commit_to(uint64_t* bar, bool both = true) {
+    if (!kPair) {
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    } else if (both) {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+    } else {
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    }
 }
 // Shared-memory matrix descriptors are passed as (low word, high word): only the low word (start
 // address and leading byte offset) varies between the MMAs of a kernel, so the issuing thread keeps
@@ -160,6 +199,19 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t 
                  "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
                  ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc) : "memory");
+}
+// The same two for a CTA pair: M = 256, each CTA supplies its 128 rows of A and its half of B's N extent.
+__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t acc) {
@@ -188,11 +240,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+__device__ __forceinline__ void tmem_st2(uint32_t taddr, uint32_t a, uint32_t b) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
+}
+// two columns, waited for
+__device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t& a, uint32_t& b) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -215,11 +269,13 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) 
 }
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N as given.
-constexpr uint32_t idesc_f16(uint32_t n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t idesc_f16(uint32_t n, uint32_t m = 128u) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 constexpr uint32_t kIdescQK = idesc_f16(kStepKeys);              // S (128 x 128): A, B both K-major
 constexpr uint32_t kIdescPV = idesc_f16(kHeadDim) | (1u << 16);  // O (128 x 128): B (= V) MN-major
+constexpr uint32_t kIdescQK2 = idesc_f16(kStepKeys, 256u);       // the same over the 256 rows of a CTA pair
+constexpr uint32_t kIdescPV2 = idesc_f16(kHeadDim, 256u) | (1u << 16);
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -333,15 +389,6 @@ __device__ __forceinline__ void mask_chunk(uint32_t* sr, int pos0, int L, int N,
         const bool vis = jt < 0 || (jt < N && ((anc >> jt) & 1ull));
         if (!vis) sr[i] = 0xff800000u;                    // -inf
     }
-}
-
-// The 128 scores of a step for one query row, TMEM -> registers: four loads, one wait.
-__device__ __forceinline__ void load_scores(uint32_t s_taddr, uint32_t (&sr)[128]) {
-    tmem_ld32(s_taddr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-    tmem_ld32(s_taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-    tmem_ld32(s_taddr + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
-    tmem_ld32(s_taddr + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
-    tmem_wait_ld();
 }
 
 // O row *= alpha for the 32 rows of this warp (rare: only when a row maximum grew by more than 2^8).
@@ -470,19 +517,28 @@ struct SegIter {
     }
 };
 
+template <bool kPair>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qmap,
                       const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128B swizzle pattern repeats every 1024 bytes of address
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sQ = smem;                                 // [2 tiles][2 d-halves][128 rows][128 B]
-    uint8_t* sK = sQ + 2 * kQTileBytes;                 // [kKStages][2 d-halves][128 keys][128 B]
-    uint8_t* sV = sK + kKStages * kTileBytes;           // [kVStages][2 d-halves][128 keys][128 B]
-    Shared* sh = reinterpret_cast<Shared*>(sV + kVStages * kTileBytes);
+    uint8_t* sQ = smem;                                 // [2 d-halves][128 rows][128 B]
+    using C = Cfg<kPair>;
+    constexpr int kStages = C::kStages, kDepth = C::kDepth, kRing = C::kRing, kTile = C::kTile, kKHalf = C::kKHalf;
+    // single: K [stage][2 d-halves][128 keys][128 B], V the same; pair: K [stage][2 d-halves][this CTA's 64 keys][128 B],
+    // V [stage][128 keys][this CTA's 64-wide d-half = 128 B]
+    uint8_t* sK = sQ + kQTileBytes;
+    uint8_t* sV = sK + kStages * kTile;
+    Shared* sh = reinterpret_cast<Shared*>(sV + kStages * kTile);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // member = row tile of the tree that this CTA owns; a pair is two consecutive members
     const int member = blockIdx.x % p.n_rp, gang = blockIdx.x / p.n_rp;
+    const int crank = kPair ? (member & 1) : 0;                     // rank in the pair; rank 0 issues the MMAs
+    const bool is_lead = crank == 0;
+    const int member0 = kPair ? (member & ~1) : member;            // first member of the pair: decides whether an item is this pair's
 
     // ---- this gang's range of steps (warp 0 computes, everybody reads)
     if (warp == 0) {
@@ -513,27 +569,47 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
 
     // ---- set-up: barriers, TMEM
     if (tid == 0) {
-        for (int i = 0; i < kRing; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_done[i], 1); }
+        // Pair form: the leader's "landed" barriers also take the relayed arrival of the partner's copies, and
+        // the barriers that the softmax warps arrive on count the warps of both CTAs.
+        const int lands = (kPair && is_lead) ? 2 : 1;
+        for (int i = 0; i < kRing; ++i) { mbar_init(&sh->kv_full[i], lands); mbar_init(&sh->kv_done[i], 1); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh->s_full[t], 1);
-            mbar_init(&sh->p_full[t], 4);               // one arrival per softmax warp
+            mbar_init(&sh->p_full[t], kPair ? 8 : 4);   // one arrival per softmax warp of the slot
             mbar_init(&sh->o_full[t], 1);
         }
+        mbar_init(&sh->epi_done, kPair ? 16 : 8);       // one arrival per softmax warp
         mbar_init(&sh->q_free, 1);
         mbar_init(&sh->drain, 1);
-        mbar_init(&sh->q_ready, 1);
+        mbar_init(&sh->q_ready, lands);
         sh->abort = 0;
+        sh->peer_abort = kPair ? cluster_addr(&sh->abort, crank ^ 1) : 0u;
+        for (int i = 0; i < 8; ++i) (&sh->eflag[0][0])[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 9) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&sh->tmem_base)), "r"(512) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (kPair) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&sh->tmem_base)), "r"(512) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&sh->tmem_base)), "r"(512) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (kPair) {
+        // both CTAs' barriers and tensor memory exist before either touches the other's
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
+    // where the softmax warps arrive: the leader's barriers
+    const uint32_t lead_p_full[2] = {kPair ? cluster_addr(&sh->p_full[0], 0) : 0u, kPair ? cluster_addr(&sh->p_full[1], 0) : 0u};
+    const uint32_t lead_epi_done = kPair ? cluster_addr(&sh->epi_done, 0) : 0u;
 
     // Registers move from the copy / MMA warpgroup (which needs few) to the softmax warpgroups:
     // 4 warps give up 168 - 72 registers per thread, 8 warps take 216 - 168 each.
@@ -545,20 +621,19 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
             SegIter it;
             it.init(sh);
             Seg sg;
-            // A segment of n steps takes n + 1 ring steps: ring step i carries the K tile of step s0 + i
-            // (i < n) and the V tile of step s0 + i - 1 (i > 0), which is what the MMA warp consumes together
-            // ([P V of the step before, scores of this step]); both land on one barrier.
+            // A segment of n steps takes n + 2 ring steps: ring step i carries the K tile of step s0 + i
+            // (i < n) and the V tile of step s0 + i - 2 (i >= 2), which is what the MMA warp consumes together
+            // ([P V of the step two back, scores of this step]); both land on one barrier.
             int rc = 0, kc = 0, vc = 0, nq = 0;          // ring steps, K tiles, V tiles, query loads issued so far
             bool ok = !p.producer_off;
             while (ok && it.next(p, sg)) {
-                if (member >= sg.rp) continue;
-                const int M = sg.N * p.G;
-                const int n_rt = (M - member * kRowsPerCta > kRowTile) ? 2 : 1;
+                if (member0 >= sg.rp) continue;
                 const int32_t* pages = p.page_table + (size_t)sg.b * p.max_pages;
                 const int n_pages_seq = (sg.L + sg.N + kPageSize - 1) / kPageSize;
                 const int n = sg.s1 - sg.s0;
-                int ids_prev[2] = {0, 0}, npg_prev = 0;
-                for (int i = 0; i <= n; ++i) {
+                int ids_a[2] = {0, 0}, npg_a = 0;        // pages of step i - 1
+                int ids_b[2] = {0, 0}, npg_b = 0;        // pages of step i - 2
+                for (int i = 0; i < n + 2; ++i) {
                     const int j = sg.s0 + i;
                     // page ids of step j (checked: they become TMA coordinates)
                     int ids[2] = {0, 0}, npg = 0;
@@ -572,127 +647,168 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
                             }
                         }
                     }
-                    // the tiles that ring step rc - 2 used are free once its MMAs have finished
-                    if (rc >= 2 && !mbar_wait(&sh->kv_done[(rc - 2) % kRing], ((rc - 2) / kRing) & 1, sh, p)) { ok = false; break; }
+                    // the tiles that ring step rc - kDepth used are free once its MMAs have finished
+                    if (rc >= kDepth &&
+                        !mbar_wait(&sh->kv_done[(rc - kDepth) % kRing], ((rc - kDepth) / kRing) & 1, sh, p)) { ok = false; break; }
                     uint64_t* full = &sh->kv_full[rc % kRing];
-                    mbar_expect_tx(full, (npg + (i > 0 ? npg_prev : 0)) * 2 * kPageHalfBytes);
-                    if (i < n) {
-                        const int kslot = kc % kKStages;
-                        for (int pi = 0; pi < npg; ++pi)
+                    const int npv = i >= 2 ? npg_b : 0;
+                    if (!kPair) {
+                        mbar_expect_tx(full, (npg + npv) * 2 * kPageHalfBytes);
+                        if (i < n) {
+                            const int kslot = kc % kStages;
+                            for (int pi = 0; pi < npg; ++pi)
+                                for (int h = 0; h < 2; ++h)
+                                    tma_load_4d(smem_u32(sK + kslot * kTile + h * kKHalf + pi * kPageHalfBytes), &kmap,
+                                                h * 64, 0, ids[pi] * p.Hkv + sg.g, sg.layer, full);
+                        }
+                        for (int pi = 0; pi < npv; ++pi)
                             for (int h = 0; h < 2; ++h)
-                                tma_load_4d(smem_u32(sK + kslot * kTileBytes + h * kTileHalfBytes + pi * kPageHalfBytes), &kmap,
-                                            h * 64, 0, ids[pi] * p.Hkv + sg.g, sg.layer, full);
-                        ++kc;
-                    }
-                    if (i > 0) {
-                        const int vslot = vc % kVStages;
-                        for (int pi = 0; pi < npg_prev; ++pi)
+                                tma_load_4d(smem_u32(sV + (vc % kStages) * kTile + h * kTileHalfBytes + pi * kPageHalfBytes), &vmap,
+                                            h * 64, 0, ids_b[pi] * p.Hkv + sg.g, sg.layer, full);
+                    } else {
+                        // this CTA's share: page `crank` of the K tile (both d-halves), d-half `crank` of the V tile (both pages)
+                        const bool my_k = i < n && crank < npg;
+                        mbar_expect_tx(full, ((my_k ? 2 : 0) + npv) * kPageHalfBytes);
+                        if (my_k)
                             for (int h = 0; h < 2; ++h)
-                                tma_load_4d(smem_u32(sV + vslot * kTileBytes + h * kTileHalfBytes + pi * kPageHalfBytes), &vmap,
-                                            h * 64, 0, ids_prev[pi] * p.Hkv + sg.g, sg.layer, full);
-                        ++vc;
+                                tma_load_4d(smem_u32(sK + (kc % kStages) * kTile + h * kKHalf), &kmap,
+                                            h * 64, 0, ids[crank] * p.Hkv + sg.g, sg.layer, full);
+                        for (int pi = 0; pi < npv; ++pi)
+                            tma_load_4d(smem_u32(sV + (vc % kStages) * kTile + pi * kPageHalfBytes), &vmap,
+                                        crank * 64, 0, ids_b[pi] * p.Hkv + sg.g, sg.layer, full);
                     }
+                    if (i < n) ++kc;
+                    if (i >= 2) ++vc;
                     ++rc;
                     if (i == 0) {
-                        // the segment's query tiles, once the previous segment's score MMAs have read theirs
+                        // the segment's query tile, once the previous segment's score MMAs have read theirs
                         if (nq > 0 && !mbar_wait(&sh->q_free, (nq - 1) & 1, sh, p)) { ok = false; break; }
-                        mbar_expect_tx(&sh->q_ready, n_rt * kQTileBytes);
-                        for (int t = 0; t < n_rt; ++t)
-                            for (int h = 0; h < 2; ++h)
-                                tma_load_5d(smem_u32(sQ + t * kQTileBytes + h * kQHalfBytes), &qmap, h * 64, 0, sg.g,
-                                            sg.n0 + (member * kRowsPerCta + t * kRowTile) / p.G, sg.layer, &sh->q_ready);
+                        // (a tile past the end of the tree, in the pair form, reads rows that are never stored)
+                        mbar_expect_tx(&sh->q_ready, kQTileBytes);
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_5d(smem_u32(sQ + h * kQHalfBytes), &qmap, h * 64, 0, sg.g,
+                                        sg.n0 + (member * kRowsPerCta) / p.G, sg.layer, &sh->q_ready);
                         ++nq;
                     }
-                    ids_prev[0] = ids[0]; ids_prev[1] = ids[1]; npg_prev = npg;
+                    ids_b[0] = ids_a[0]; ids_b[1] = ids_a[1]; npg_b = npg_a;
+                    ids_a[0] = ids[0]; ids_a[1] = ids[1]; npg_a = npg;
                 }
             }
             if (sh->abort) {
                 // drain: every issued copy must land before the CTA may exit
-                for (int n = max(0, rc - 2); n < rc; ++n)
+                for (int n = max(0, rc - kDepth); n < rc; ++n)
                     mbar_wait_quiet(&sh->kv_full[n % kRing], (n / kRing) & 1, p.wait_cycles);
                 if (nq > 0) mbar_wait_quiet(&sh->q_ready, (nq - 1) & 1, p.wait_cycles);
             }
         }
+    } else if (warp == 10) {
+        // =========================== relay (pair form, second CTA) ===========================
+        // The MMA thread of the leader waits on the leader's barriers only; what lands in this CTA is passed on
+        // to them, in the order in which the MMA thread waits.
+        if (kPair && !is_lead && lane == 0) {
+            SegIter it;
+            it.init(sh);
+            Seg sg;
+            int rc = 0, nq = 0;
+            bool ok = true;
+            while (ok && it.next(p, sg)) {
+                if (member0 >= sg.rp) continue;
+                const int n = sg.s1 - sg.s0;
+                for (int i = 0; ok && i < n + 2; ++i) {
+                    if (i == 0) {
+                        ok = mbar_wait(&sh->q_ready, nq & 1, sh, p);
+                        if (!ok) break;
+                        ++nq;
+                        mbar_arrive_cluster(cluster_addr(&sh->q_ready, 0));
+                    }
+                    ok = mbar_wait(&sh->kv_full[rc % kRing], (rc / kRing) & 1, sh, p);
+                    if (!ok) break;
+                    mbar_arrive_cluster(cluster_addr(&sh->kv_full[rc % kRing], 0));
+                    ++rc;
+                }
+            }
+        }
     } else if (warp == 9) {
         // =========================== MMA issuer ===========================
-        // One thread issues for both row tiles, in blocks [P V of step j-1, scores of step j] per tile:
-        // a tile's block runs on the tensor pipe while the other tile's warpgroup is in its softmax, and
-        // the blocks of the two tiles never interleave (two issuers would finish both tiles' scores at
-        // the same moment and leave the pipe idle during both softmaxes).  The whole instruction stream
-        // sits in one single-thread region: a predicated branch around every MMA costs more issue time
-        // than the MMA takes to execute.
-        if (lane == 0) {
+        // One thread issues for both slots, in blocks [P V of step i-2, scores of step i]: step i belongs to
+        // slot i & 1, so a slot's block runs on the tensor pipe while the other slot's warpgroup is in its
+        // softmax, and the blocks never interleave.  The whole instruction stream sits in one single-thread
+        // region: a predicated branch around every MMA costs more issue time than the MMA takes to execute.
+        if (lane == 0 && is_lead) {
             // descriptors differ only in their 14-bit start-address field (bytes >> 4); shared memory ends below 256 KB
+            // (pair form: the same offsets hold the partner's parts in its shared memory)
             const uint32_t dq = desc_lo(smem_u32(sQ), 16);
             const uint32_t dk = desc_lo(smem_u32(sK), 16);
             const uint32_t dv = desc_lo(smem_u32(sV), kTileHalfBytes);
             auto issue_qk = [&](int t, int slot) {
-                // S_t = Q_t K^T: 8 slices of K = 16 over d = 128 (4 per 64-wide half)
-                const uint32_t dqt = dq + ((t * kQTileBytes) >> 4);
-                const uint32_t dks = dk + ((slot * kTileBytes) >> 4);
+                // S_t = Q K^T: 8 slices of K = 16 over d = 128 (4 per 64-wide half)
+                const uint32_t dks = dk + ((slot * kTile) >> 4);
                 const uint32_t s_tmem = tmem + t * 128;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ss(s_tmem, dqt + (((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4),
-                           dks + (((ks >> 2) * kTileHalfBytes + (ks & 3) * 32) >> 4), kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t a = dq + (((ks >> 2) * kQHalfBytes + (ks & 3) * 32) >> 4);
+                    const uint32_t b = dks + (((ks >> 2) * kKHalf + (ks & 3) * 32) >> 4);
+                    if (kPair) mma2_ss(s_tmem, a, b, kDescHi, kIdescQK2, ks > 0 ? 1u : 0u);
+                    else mma_ss(s_tmem, a, b, kDescHi, kIdescQK, ks > 0 ? 1u : 0u);
+                }
             };
             auto issue_pv = [&](int t, int slot, bool first) {
                 // O_t += P_t V: 8 slices of K = 16 keys; P in TMEM (8 columns per slice), V MN-major
-                const uint32_t dvs = dv + ((slot * kTileBytes) >> 4);
+                const uint32_t dvs = dv + ((slot * kTile) >> 4);
                 const uint32_t s_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(o_tmem, s_tmem + ks * 8, dvs + ((ks * 2048) >> 4), kDescHi, kIdescPV, (first && ks == 0) ? 0u : 1u);
+                for (int ks = 0; ks < 8; ++ks) {
+                    if (kPair) mma2_ts(o_tmem, s_tmem + ks * 8, dvs + ((ks * 2048) >> 4), kDescHi, kIdescPV2, (first && ks == 0) ? 0u : 1u);
+                    else mma_ts(o_tmem, s_tmem + ks * 8, dvs + ((ks * 2048) >> 4), kDescHi, kIdescPV, (first && ks == 0) ? 0u : 1u);
+                }
             };
             SegIter it;
             it.init(sh);
             Seg sg;
-            int rc = 0, kc = 0, vc = 0, nq = 0;             // ring steps, K tiles, V tiles consumed; segments started
-            int np[2] = {0, 0};                             // steps of each row tile whose probabilities were consumed
+            int rc = 0, kc = 0, vc = 0, nseg = 0;           // ring steps, K tiles, V tiles consumed; segments started
+            int np[2] = {0, 0};                             // steps of each slot whose probabilities were consumed
             bool ok = true;
             // Every synchronisation instruction costs this thread a couple of hundred clocks, during which
             // at most a few queued MMAs keep the pipe busy: the loop holds as few of them as the protocol
-            // allows (one wait and one commit per ring step for the tiles, one of each per row tile).
+            // allows (one wait and one commit per ring step for the tiles, one of each for the step's slot).
             while (ok && it.next(p, sg)) {
-                if (member >= sg.rp) continue;
-                const int n_rt = (sg.N * p.G - member * kRowsPerCta > kRowTile) ? 2 : 1;
-                const int s0 = sg.s0, s1 = sg.s1;
-                ok = mbar_wait(&sh->q_ready, nq & 1, sh, p);
-                ++nq;
-                // ring step: the P V products of step j - 1 (when j > s0) and the scores of step j (when j < s1)
-                for (int j = s0; ok && j <= s1; ++j) {
-                    ok = mbar_wait(&sh->kv_full[rc % kRing], (rc / kRing) & 1, sh, p);
+                if (member0 >= sg.rp) continue;
+                const int n = sg.s1 - sg.s0;
+                ok = mbar_wait<kPair>(&sh->q_ready, nseg & 1, sh, p);
+                for (int i = 0; ok && i < n + 2; ++i) {
+                    ok = mbar_wait<kPair>(&sh->kv_full[rc % kRing], (rc / kRing) & 1, sh, p);
                     if (!ok) break;
-                    const int kslot = kc % kKStages, vslot = vc % kVStages;
-                    if (j < s1) ++kc;
-                    if (j > s0) ++vc;
-#pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        if (t < n_rt) {
-                            if (j > s0) {
-                                // (the warpgroup zeroed the V rows past the end of the sequence before it arrived)
-                                ok = mbar_wait(&sh->p_full[t], np[t] & 1, sh, p);
-                                if (!ok) break;
-                                ++np[t];
-                                tc_fence_after();
-                                issue_pv(t, vslot, j - 1 == s0);
-                                if (j == s1) tc_commit(true, &sh->o_full[t]);   // every MMA of this tile's segment has been issued
-                            }
-                            if (j < s1) {
-                                issue_qk(t, kslot);
-                                tc_commit(true, &sh->s_full[t]);
-                            }
+                    const int t = i & 1;
+                    if (i >= 2) {
+                        // (the warpgroup zeroed the V rows past the end of the sequence before it arrived)
+                        ok = mbar_wait<kPair>(&sh->p_full[t], np[t] & 1, sh, p);
+                        if (!ok) break;
+                        ++np[t];
+                        // the segment's first P V products overwrite both accumulators, which the softmax warps
+                        // read in the epilogue of the segment before
+                        if (i == 2 && nseg > 0) {
+                            ok = mbar_wait<kPair>(&sh->epi_done, (nseg - 1) & 1, sh, p);
+                            if (!ok) break;
                         }
+                        tc_fence_after();
+                        issue_pv(t, vc % kStages, i < 4);
+                        ++vc;
+                        if (i >= n) tc_commit_to<kPair>(&sh->o_full[t]);    // the slot's last step of the segment
                     }
-                    if (!ok) break;
-                    tc_commit(true, &sh->kv_done[rc % kRing]);
+                    if (i < n) {
+                        issue_qk(t, kc % kStages);
+                        ++kc;
+                        tc_commit_to<kPair>(&sh->s_full[t]);
+                    }
+                    tc_commit_to<kPair>(&sh->kv_done[rc % kRing]);
                     ++rc;
-                    if (j == s1 - 1) tc_commit(true, &sh->q_free);          // the segment's last score MMAs read the query tiles
+                    if (i == n - 1) tc_commit_to<kPair>(&sh->q_free);   // the segment's last score MMAs read the query tile
                 }
+                ++nseg;
             }
             if (!ok) {
                 // abort: everything this thread has issued must retire before the TMEM and the tiles go away
-                tc_commit(true, &sh->drain);
+                tc_commit_to<kPair>(&sh->drain, false);
                 mbar_wait_quiet(&sh->drain, 0, p.wait_cycles);
             }
         }
@@ -701,28 +817,32 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== softmax warpgroups ===========================
-        const int t = warp >> 2;                        // row tile of this warpgroup
+        // Warpgroup t owns slot t: the steps s0 + t, s0 + t + 2, ... of a segment, with its own score tile S_t,
+        // accumulator O_t and running (reference, sum) per row; one thread per query row.  In the epilogue the
+        // two slots are combined, warpgroup t taking the output columns [64t, 64t + 64).
+        const int t = warp >> 2, q = warp & 3;
         const int r = tid & 127;                        // row inside the tile == TMEM lane
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const uint32_t s_taddr = tmem + lane_base + t * 128;
         const uint32_t o_taddr = tmem + lane_base + 256 + t * 128;
         SegIter it;
         it.init(sh);
         Seg sg;
-        int nsteps = 0, nseg = 0;                       // steps / segments this row tile has been through
+        int nst = 0;                                    // steps this slot has been through
+        int nseg = 0, nseg1 = 0;                        // segments so far; those in which slot 1 had steps
         int rc0 = 0, vc0 = 0;                           // ring steps / V tiles of the CTA before the current segment
         bool ok = true;
         while (ok && it.next(p, sg)) {
-            if (member >= sg.rp) continue;
+            if (member0 >= sg.rp) continue;
             const int M = sg.N * p.G;
-            const int rc_seg = rc0, vc_seg = vc0;       // this segment's first ring step / V tile
-            rc0 += sg.s1 - sg.s0 + 1;
-            vc0 += sg.s1 - sg.s0;
-            if (t == 1 && M - member * kRowsPerCta <= kRowTile) continue;
-            const int R = member * kRowsPerCta + t * kRowTile + r;
+            const int n = sg.s1 - sg.s0;
+            const int rc_seg = rc0, vc_seg = vc0;       // this segment's first ring step / V tile (= steps so far)
+            rc0 += n + 2;
+            vc0 += n;
+            const int R = member * kRowsPerCta + r;
             const bool row_ok = R < M;
             const int node = row_ok ? R / p.G : 0;
-            const bool warp_live = member * kRowsPerCta + t * kRowTile + (warp & 3) * 32 < M;
+            const bool warp_live = member * kRowsPerCta + q * 32 < M;
             uint64_t anc = 0;
             if (sg.s1 * kStepKeys > sg.L && row_ok) {
                 // the segment reaches the tree part: this row's ancestor bitset (the G rows of a node
@@ -732,22 +852,24 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
                 if (bad) { report_status(p.status, SAGE_STATUS_BAD_TREE); anc = 1ull << node; }
             }
             float m_ref = -INFINITY, l_sum = 0.f;
-            for (int j = sg.s0; j < sg.s1; ++j) {
-                ok = mbar_wait(&sh->s_full[t], nsteps & 1, sh, p);
+            for (int i = t; i < n; i += 2) {
+                const int j = sg.s0 + i;
+                ok = mbar_wait(&sh->s_full[t], nst & 1, sh, p);
                 if (!ok) break;
+                ++nst;
                 const int valid = sg.L + sg.N - j * kStepKeys;      // keys of this step that exist
                 if (valid < kStepKeys) {
                     // V rows past the end of the sequence may hold anything (a missing second page was not even
                     // copied): zero them so that 0 * V stays 0.  Each warp of the warpgroup takes a quarter of
-                    // the rows (both warpgroups write the same zeros); the writes are ordered before this
-                    // warp's arrival, which the P V product waits for.  The V tile of step j lands with ring
-                    // step j - s0 + 1 of the segment.
-                    const int rcv = rc_seg + (j - sg.s0) + 1;
+                    // the rows; the writes are ordered before this warp's arrival, which the P V product waits
+                    // for.  The V tile of step s0 + i lands with ring step i + 2 of the segment.
+                    const int rcv = rc_seg + i + 2;
                     ok = mbar_wait(&sh->kv_full[rcv % kRing], (rcv / kRing) & 1, sh, p);
                     if (!ok) break;
-                    uint8_t* vb = sV + ((vc_seg + (j - sg.s0)) % kVStages) * kTileBytes;
-                    for (int c = (warp & 3) * 32 + lane; c < (kStepKeys - valid) * 16; c += 128) {
-                        const int vr = valid + c / 16, ch = c % 16;
+                    uint8_t* vb = sV + ((vc_seg + i) % kStages) * kTile;
+                    constexpr int kChunks = kPair ? 8 : 16;             // 16-byte chunks of a V row held by this CTA
+                    for (int c = q * 32 + lane; c < (kStepKeys - valid) * kChunks; c += 128) {
+                        const int vr = valid + c / kChunks, ch = c % kChunks;
                         *reinterpret_cast<uint4*>(vb + (ch >> 3) * kTileHalfBytes + vr * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -755,23 +877,30 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
                 if (!warp_live) {
                     // none of this warp's 32 rows exists (ragged last tile): keep the barrier protocol
                     // going, leave the probabilities of these rows as they are; their outputs are never stored
-                    ++nsteps;
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&sh->p_full[t]);
+                    if (lane == 0) {
+                    if (kPair && !is_lead) mbar_arrive_cluster(lead_p_full[t]);
+                    else mbar_arrive(&sh->p_full[t]);
+                }
                     continue;
                 }
                 tc_fence_after();
                 const int pos0 = j * kStepKeys;
                 const bool masked = pos0 + kStepKeys > sg.L;     // reaches into the tree part (or past the end)
+                // the 128 scores of the row: the second half is still on its way while the first is looked at
                 uint32_t sr[128];
-                load_scores(s_taddr, sr);
-                if (masked) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) mask_chunk(sr + 32 * c, pos0 + 32 * c, sg.L, sg.N, anc);
-                }
+                tmem_ld32(s_taddr, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                tmem_ld32(s_taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                tmem_wait_ld();
+                tmem_ld32(s_taddr + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+                tmem_ld32(s_taddr + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
                 float mx = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) max_chunk(sr + 32 * c, mx);
+                for (int c = 0; c < 4; ++c) {
+                    if (c == 2) tmem_wait_ld();
+                    if (masked) mask_chunk(sr + 32 * c, pos0 + 32 * c, sg.L, sg.N, anc);
+                    max_chunk(sr + 32 * c, mx);
+                }
                 // lazy rescale: the reference moves only when the row max grew by more than 2^8 over it
                 const float m_cand = mx * p.scale_log2;
                 const bool grow = m_cand > m_ref + 8.0f;
@@ -780,85 +909,160 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
                     alpha = fast_exp2(m_ref - m_cand);              // 0 when m_ref was -inf
                     m_ref = m_cand;
                 }
-                // O_t *= alpha.  The P V product of the step before has finished: the scores of this step were
-                // issued after it, and their completion is what this warp waited for above.
-                if (j > sg.s0 && __any_sync(0xffffffffu, grow)) rescale_o_rows(o_taddr, alpha);
+                // O_t *= alpha.  The slot's P V product of two steps back has finished: the scores of this step
+                // were issued after it, and their completion is what this warp waited for above.
+                if (i >= 2 && __any_sync(0xffffffffu, grow)) rescale_o_rows(o_taddr, alpha);
                 const float neg_ref = (m_ref == -INFINITY) ? 0.f : -m_ref;
                 // probabilities, packed to bf16 in place: chunk c (32 scores) leaves its 16 words at sr[16c ..]
+                // (P goes over the first 64 columns of S_t, the first half as soon as it is there)
                 uint64_t acc[2] = {0ull, 0ull};
                 if (masked) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) exp_chunk<0>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);   // may hold -inf
+                    for (int c = 0; c < 4; ++c) {
+                        exp_chunk<0>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);   // may hold -inf
+                        if (c == 1) tmem_st32(s_taddr, sr);
+                    }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) exp_chunk<SAGE_EXP2_FMA_PAIRS>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);
+                    for (int c = 0; c < 4; ++c) {
+                        exp_chunk<SAGE_EXP2_FMA_PAIRS>(sr + 32 * c, p.scale_log2, neg_ref, sr + 16 * c, acc);
+                        if (c == 1) tmem_st32(s_taddr, sr);
+                    }
                 }
+                tmem_st32(s_taddr + 32, sr + 32);
                 float sum_a, sum_b;
                 f2_unpack(f2_add(acc[0], acc[1]), sum_a, sum_b);
                 l_sum = l_sum * alpha + (sum_a + sum_b);
-                uint32_t* pk = sr;
-                tmem_st32(s_taddr, pk);                 // P over the first 64 columns of S_t
-                tmem_st32(s_taddr + 32, pk + 32);
                 tmem_wait_st();
                 tc_fence_before();
-                ++nsteps;
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh->p_full[t]);
+                if (lane == 0) {
+                    if (kPair && !is_lead) mbar_arrive_cluster(lead_p_full[t]);
+                    else mbar_arrive(&sh->p_full[t]);
+                }
             }
             if (!ok) break;
-            // ---- epilogue: O_t / l -> bf16 output, or unnormalised partials for the merge
-            ok = mbar_wait(&sh->o_full[t], nseg & 1, sh, p);
+            // ---- epilogue: the two slots combined, then O / l -> bf16 output, or unnormalised partials for the merge
+            const bool has1 = n >= 2;                   // slot 1 took part in this segment
+            ok = mbar_wait(&sh->o_full[0], nseg & 1, sh, p);
+            if (ok && has1) ok = mbar_wait(&sh->o_full[1], nseg1 & 1, sh, p);
+            const uint32_t eseq = (uint32_t)nseg + 1u;
             ++nseg;
+            if (has1) ++nseg1;
             if (!ok) break;
-            tc_fence_after();
-            const bool whole = (sg.s0 == 0 && sg.s1 == sg.steps);
-            const float inv = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
-            float* po = nullptr;
-            __nv_bfloat16* oo = nullptr;
-            if (whole) {
-                const size_t row = (size_t)(sg.n0 + node) * p.Hq + sg.g * p.G + (row_ok ? R % p.G : 0);
-                oo = p.out + ((size_t)sg.layer * p.sum_nodes * p.Hq + row) * kHeadDim;
-            } else {
-                const size_t pr = (((size_t)gang * 2 + (sg.at_range_begin ? 0 : 1)) * p.n_rp + member) * kRowsPerCta +
-                                  t * kRowTile + r;
-                po = p.part_o + pr * kHeadDim;
-                if (row_ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = l_sum; }
-            }
             if (warp_live) {
+                tc_fence_after();
+                // this thread's 64 columns of both accumulators, 32 at a time
+                const uint32_t o0 = tmem + lane_base + 256 + 64 * t, o1 = o0 + 128;
+                uint32_t oa[32], ob[32];
+                tmem_ld32(o0, oa);
+                if (has1) tmem_ld32(o1, ob);
+                tmem_wait_ld();
+                // The row's (reference, sum) of this slot goes to the other warpgroup through two columns of O_t
+                // that this thread has just read and nobody else reads: columns 64t and 64t + 1.
+                tmem_st2(o_taddr + 64 * t, __float_as_uint(m_ref), __float_as_uint(l_sum));
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence_block();
+                    sh->eflag[t][q] = eseq;
+                }
+                // bounded wait for the partner warp (same rows, other slot)
+                {
+                    volatile uint32_t* flag = &sh->eflag[1 - t][q];
+                    bool seen = (*flag == eseq);
+                    if (!seen) {
+                        const long long t0 = clock64();
+                        while (true) {
+                            for (int k = 0; k < 64 && !seen; ++k) seen = (*flag == eseq);
+                            if (seen || sh->abort) break;
+                            if (clock64() - t0 > p.wait_cycles) {
+                                raise_abort(sh);
+                                report_status(p.status, SAGE_STATUS_TIMEOUT);
+                                break;
+                            }
+                        }
+                    }
+                    ok = __all_sync(0xffffffffu, seen);
+                }
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t pm, pl;
+                tmem_ld2(tmem + lane_base + 256 + (1 - t) * 128 + 64 * (1 - t), pm, pl);
+                const float m_o = __uint_as_float(pm), l_o = __uint_as_float(pl);
+                // weights of the two slots under the common reference (a slot without visible keys has l = 0)
+                const float m_all = fmaxf(l_sum > 0.f ? m_ref : -INFINITY, l_o > 0.f ? m_o : -INFINITY);
+                const float w_me = l_sum > 0.f ? fast_exp2(m_ref - m_all) : 0.f;
+                const float w_ot = l_o > 0.f ? fast_exp2(m_o - m_all) : 0.f;
+                const float l_all = l_sum * w_me + l_o * w_ot;
+                const bool whole = (sg.s0 == 0 && sg.s1 == sg.steps);
+                // factors of O_0 and O_1: the slot weights, and 1 / l for a finished row
+                const float inv = whole ? ((l_all > 0.f) ? 1.0f / l_all : 0.f) : 1.0f;
+                const float f0 = (t == 0 ? w_me : w_ot) * inv, f1 = has1 ? (t == 0 ? w_ot : w_me) * inv : 0.f;
+                __nv_bfloat16* oo = nullptr;
+                float* po = nullptr;
+                if (whole) {
+                    const size_t row = (size_t)(sg.n0 + node) * p.Hq + sg.g * p.G + (row_ok ? R % p.G : 0);
+                    oo = p.out + ((size_t)sg.layer * p.sum_nodes * p.Hq + row) * kHeadDim + 64 * t;
+                } else {
+                    const size_t pr = (((size_t)gang * 2 + (sg.at_range_begin ? 0 : 1)) * p.n_rp + member) * kRowsPerCta + r;
+                    po = p.part_o + pr * kHeadDim + 64 * t;
+                    if (t == 0 && row_ok) { p.part_ml[pr * 2] = m_all; p.part_ml[pr * 2 + 1] = l_all; }
+                }
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t orr[32];
-                    tmem_ld32(o_taddr + c * 32, orr);
-                    tmem_wait_ld();
+                for (int c = 0; c < 2; ++c) {
+                    if (c == 1) {
+                        tmem_ld32(o0 + 32, oa);
+                        if (has1) tmem_ld32(o1 + 32, ob);
+                        tmem_wait_ld();
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        float v = __uint_as_float(oa[i]) * f0;
+                        if (has1) v = fmaf(__uint_as_float(ob[i]), f1, v);
+                        oa[i] = __float_as_uint(v);
+                    }
                     if (row_ok) {
-                        if (oo) {
+                        if (whole) {
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 uint4 v;
-                                v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+                                v.x = pack_bf16(__uint_as_float(oa[8 * i + 0]), __uint_as_float(oa[8 * i + 1]));
+                                v.y = pack_bf16(__uint_as_float(oa[8 * i + 2]), __uint_as_float(oa[8 * i + 3]));
+                                v.z = pack_bf16(__uint_as_float(oa[8 * i + 4]), __uint_as_float(oa[8 * i + 5]));
+                                v.w = pack_bf16(__uint_as_float(oa[8 * i + 6]), __uint_as_float(oa[8 * i + 7]));
                                 *reinterpret_cast<uint4*>(oo + c * 32 + i * 8) = v;
                             }
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
-                                *reinterpret_cast<uint4*>(po + c * 32 + i * 4) =
-                                    make_uint4(orr[4 * i], orr[4 * i + 1], orr[4 * i + 2], orr[4 * i + 3]);
+                                *reinterpret_cast<uint4*>(po + c * 32 + i * 4) = make_uint4(oa[4 * i], oa[4 * i + 1], oa[4 * i + 2], oa[4 * i + 3]);
                         }
                     }
                 }
             }
-            tc_fence_before();                          // the next segment's first P V overwrites O_t
+            tc_fence_before();                          // the next segment's first P V products overwrite O_0 and O_1
+            __syncwarp();
+            if (lane == 0) {
+                if (kPair && !is_lead) mbar_arrive_cluster(lead_epi_done);
+                else mbar_arrive(&sh->epi_done);
+            }
         }
     }
     // ---- teardown: every role is past its last TMEM access
     tc_fence_before();
     __syncthreads();
+    if (kPair) {
+        // neither CTA leaves (or frees tensor memory) while the other may still arrive on its barriers, raise
+        // its abort flag, or run MMAs that write its tensor memory
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
     if (warp == 9) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+        if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     }
 }
 
@@ -1036,14 +1240,15 @@ static int resident_ctas() {
     }
     return cached[dev];
 }
-static int row_pairs(int sum_nodes, int G) {
+// Row tiles of the largest tree the launch can hold.
+static int row_tiles(int sum_nodes, int G) {
     const int n = sum_nodes < SAGE_MAX_NODES ? sum_nodes : SAGE_MAX_NODES;      // a tree has at most that many nodes
-    return (n * G + kRowsPerCta - 1) / kRowsPerCta;
+    return (n * G + kRowTile - 1) / kRowTile;
 }
 
 static long long g_wait_cycles = kWaitCyclesDefault;
 static int g_producer_off = 0;
-static int g_schedule = 0;     // 0: chosen per launch, 1: streaming, 2: split
+static int g_schedule = 0;     // 0: chosen per launch, 1: streaming, 2: split, 3: streaming with CTA pairs
 
 // The split schedule (tree_attention_split.cu).
 namespace split {
@@ -1054,18 +1259,36 @@ int launch(const void* q, int n_layers, int n_pages, const int32_t* page_table, 
            int producer_off, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream);
 }  // namespace split
 
-// Which schedule runs a launch.  The streaming schedule (this file) wins where the work is HBM-bound and
-// long: trees of up to 256 query rows per KV head (one thread block per gang, nothing idles) with at least
-// `kStreamMinSteps` 128-key steps for every SM.  Tensor-bound trees (a gang's second block would mostly
-// repeat the first one's waits) and short launches (single layers, short contexts: fixed costs dominate)
-// go to the split schedule.
+// The streaming schedule for trees of more than one row tile (tree_attention_rows.cu).
+namespace rows {
+size_t workspace_size(int n_ctas);
+int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+           const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
+           int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
+           int producer_off, const CUtensorMap& qmap, const CUtensorMap& kmap, const CUtensorMap& vmap,
+           cudaStream_t stream);
+}  // namespace rows
+
+// Which schedule runs a launch.
+//   streaming: persistent CTAs that walk equal ranges of 128-key steps.  One row tile (up to 128 query rows
+//     per KV head): the kernel of this file, single form, which is HBM-bound.  More: two row tiles per CTA
+//     (tree_attention_rows.cu); chosen up to 256 rows, where one CTA holds the whole tree and nothing is read twice.
+//   split: grid over (context slice, row pair, layer x sequence x KV head), 64-key steps: wins where the
+//     work is tensor-bound (more than 256 rows) and where a launch is too short to give every SM a long
+//     stream (single layers, short contexts: fixed costs dominate).
+//   pairs: the kernel of this file in its pair form; measured slower than the others everywhere (the
+//     hand-overs between the two CTAs lengthen the per-step dependency chain), so never chosen, only forced.
+enum Schedule { kAlternating, kRows, kSplit, kPairs };
 constexpr int kStreamMinSteps = 16;
-static bool use_streaming(int n_layers, int batch, int sum_nodes, int n_kv_heads, int G, int max_pages_per_seq) {
-    if (g_schedule == 1) return true;
-    if (g_schedule == 2) return false;
-    if (row_pairs(sum_nodes, G) > 1) return false;
+static Schedule pick_schedule(int n_layers, int batch, int sum_nodes, int n_kv_heads, int G, int max_pages_per_seq) {
+    const int tiles = row_tiles(sum_nodes, G);
+    if (g_schedule == 1) return tiles == 1 ? kAlternating : kRows;
+    if (g_schedule == 2) return kSplit;
+    if (g_schedule == 3) return tiles == 1 ? kAlternating : kPairs;
+    if (tiles > 2) return kSplit;
     const long long steps = (long long)n_layers * batch * n_kv_heads * ((max_pages_per_seq + 1) / 2);   // upper bound
-    return steps >= (long long)kStreamMinSteps * resident_ctas();
+    if (steps < (long long)kStreamMinSteps * resident_ctas()) return kSplit;
+    return tiles == 1 ? kAlternating : kRows;
 }
 
 }  // namespace sage
@@ -1078,10 +1301,12 @@ extern "C" size_t sage_tree_attention_workspace_size(int n_layers, int batch, in
         n_q_heads % n_kv_heads)
         return 0;
     (void)head_dim;
-    // streaming schedule: two partial slots (head and tail of its range) per resident CTA, independent of the
-    // problem size; split schedule: one partial per context slice.  Either may run, so the larger is asked for.
-    const size_t streaming = (size_t)resident_ctas() * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float);
+    // streaming schedules: two partial slots (head and tail of its range) per resident CTA, independent of the
+    // problem size; split schedule: one partial per context slice.  Any may run, so the largest is asked for.
+    const size_t alternating = (size_t)resident_ctas() * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float);
+    const size_t rows_ws = rows::workspace_size(resident_ctas());
     const size_t split_ws = split::workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads, max_pages_per_seq);
+    const size_t streaming = alternating > rows_ws ? alternating : rows_ws;
     return streaming > split_ws ? streaming : split_ws;
 }
 
@@ -1090,7 +1315,7 @@ extern "C" void sage_debug_attention_waits(long long wait_cycles, int producer_o
     g_producer_off = producer_off ? 1 : 0;
 }
 
-extern "C" void sage_debug_attention_schedule(int schedule) { g_schedule = (schedule == 1 || schedule == 2) ? schedule : 0; }
+extern "C" void sage_debug_attention_schedule(int schedule) { g_schedule = (schedule >= 1 && schedule <= 3) ? schedule : 0; }
 
 extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void* v_pool, int64_t layer_stride_elems,
                                    int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
@@ -1116,21 +1341,27 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     const size_t need = sage_tree_attention_workspace_size(n_layers, batch, sum_nodes, n_q_heads, n_kv_heads,
                                                            head_dim, max_pages_per_seq);
     if (!ws || ws_bytes < need || ((uintptr_t)ws & 15)) return SAGE_ERR_WORKSPACE;
-    if ((long long)n_layers * batch * n_kv_heads > 65535 &&
-        !use_streaming(n_layers, batch, sum_nodes, n_kv_heads, G, max_pages_per_seq))
-        return SAGE_ERR_UNSUPPORTED;                    // grid limit of the split schedule
-    if (!use_streaming(n_layers, batch, sum_nodes, n_kv_heads, G, max_pages_per_seq)) {
-        CUtensorMap kmap, vmap;
-        if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
-            !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
-            return SAGE_ERR_CUDA;
+    const Schedule sched = pick_schedule(n_layers, batch, sum_nodes, n_kv_heads, G, max_pages_per_seq);
+    if (sched == kSplit && (long long)n_layers * batch * n_kv_heads > 65535) return SAGE_ERR_UNSUPPORTED;    // its grid limit
+    CUtensorMap qmap, kmap, vmap;
+    if (!make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
+        !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
+        return SAGE_ERR_CUDA;
+    if (sched == kSplit)
         return split::launch(q, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent, node_offsets, batch,
                              sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status, g_wait_cycles, g_producer_off,
                              kmap, vmap, as_stream(stream));
-    }
+    if (!make_q_map(&qmap, q, n_layers, sum_nodes, n_kv_heads, G)) return SAGE_ERR_CUDA;
+    if (sched == kRows)
+        return rows::launch(resident_ctas(), n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent,
+                            node_offsets, batch, sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status,
+                            g_wait_cycles, g_producer_off, qmap, kmap, vmap, as_stream(stream));
     const int n_ctas = resident_ctas();
     AttnParams p{};
-    p.n_rp = row_pairs(sum_nodes, G);
+    // one row tile: single CTAs; more (pair form only): CTA pairs, two row tiles each
+    const int tiles = row_tiles(sum_nodes, G);
+    const bool pair = sched == kPairs;
+    p.n_rp = pair ? 2 * ((tiles + 1) / 2) : 1;
     p.n_gangs = n_ctas / p.n_rp;
     p.out = (__nv_bfloat16*)out;
     p.part_o = (float*)ws;
@@ -1143,22 +1374,33 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     p.wait_cycles = g_wait_cycles;
     p.producer_off = g_producer_off;
 
-    CUtensorMap qmap, kmap, vmap;
-    if (!make_q_map(&qmap, q, n_layers, sum_nodes, n_kv_heads, G) ||
-        !make_pool_map(&kmap, k_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems) ||
-        !make_pool_map(&vmap, v_pool, n_layers, n_pages, n_kv_heads, layer_stride_elems))
-        return SAGE_ERR_CUDA;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SAGE_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(tree_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(tree_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return SAGE_ERR_CUDA;
         attr_set[dev] = true;
     }
-    tree_attention_kernel<<<p.n_gangs * p.n_rp, kAttnThreads, kSmemBytes, as_stream(stream)>>>(p, qmap, kmap, vmap);
+    if (pair) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(p.n_gangs * p.n_rp));
+        cfg.blockDim = dim3(kAttnThreads);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = as_stream(stream);
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, tree_attention_kernel<true>, p, qmap, kmap, vmap) != cudaSuccess) return SAGE_ERR_CUDA;
+    } else {
+        tree_attention_kernel<false><<<p.n_gangs * p.n_rp, kAttnThreads, kSmemBytes, as_stream(stream)>>>(p, qmap, kmap, vmap);
+    }
     if (p.n_gangs > 1) {
         dim3 mg((unsigned)(p.n_gangs - 1), (unsigned)((p.n_rp * kRowsPerCta + 31) / 32));
         attention_merge_kernel<<<mg, 256, 0, as_stream(stream)>>>(p);

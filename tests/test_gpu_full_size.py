@@ -23,11 +23,11 @@ N_LAYERS, L, N, N_VISUAL = 80, 16384, 60, 32 * 196
 SAMPLED_LAYERS = (0, 37, 79)
 
 
-def _build():
+def _build(n_nodes=N, shape=(3, 10)):
     dev = torch.device("cuda")
     gen = torch.Generator(device=dev)
     gen.manual_seed(523000 + 4000 + 77)
-    used = (L + N + P - 1) // P
+    used = (L + n_nodes + P - 1) // P
     n_pages = int(np.ceil(used * 1.125))
     perm = _rng(4, 1).permutation(n_pages)[:used].astype(np.int32)
     k = torch.empty((N_LAYERS, n_pages, HKV, P, D), dtype=torch.bfloat16, device=dev)
@@ -37,13 +37,13 @@ def _build():
         for layer in range(N_LAYERS):
             pool[layer].normal_(generator=gen)
             pool[layer, vis] *= 1.5
-    q = torch.empty((N_LAYERS, N, HQ, D), dtype=torch.bfloat16, device=dev).normal_(generator=gen)
-    tree = make_template(3, 10, N)
+    q = torch.empty((N_LAYERS, n_nodes, HQ, D), dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+    tree = make_template(shape[0], shape[1], n_nodes)
     return dict(k=k, v=v, q=q, perm=perm, tree=tree, page_table=dev_i32(perm.reshape(1, -1)),
-                seq_len=dev_i32([L]), parent=dev_i32(tree["parent"]), offs=dev_i32([0, N]))
+                seq_len=dev_i32([L]), parent=dev_i32(tree["parent"]), offs=dev_i32([0, n_nodes]))
 
 
-@pytest.mark.parametrize("schedule", [0, 1], ids=["as_benchmarked", "streaming"])
+@pytest.mark.parametrize("schedule", [0, 1, 3], ids=["as_benchmarked", "streaming", "pairs"])
 def test_attention_80_layers_sampled_layers_match_the_oracle_and_all_outputs_are_finite(schedule):
     w = _build()
     sage.sage_debug_attention_schedule(schedule)
@@ -55,6 +55,25 @@ def test_attention_80_layers_sampled_layers_match_the_oracle_and_all_outputs_are
     assert int(st.item()) == 0, sage.status_string(int(st.item()))
     assert bool(torch.isfinite(out.float()).all())
     offs = np.array([0, N], np.int32)
+    for layer in SAMPLED_LAYERS:
+        want = oracle.tree_attention(host_bits(w["q"][layer]), host_bits(w["k"][layer]), host_bits(w["v"][layer]),
+                                     w["perm"].reshape(1, -1), np.array([L], np.int32), w["tree"]["parent"], offs,
+                                     HQ, HKV, D, P, 1.0 / np.sqrt(D))
+        check_attention(host_bits(out[layer]), want)
+
+
+@pytest.mark.parametrize("n_nodes,shape", [(16, (8, 2)), (24, (8, 2))], ids=["16_nodes", "24_nodes"])
+def test_attention_80_layers_deep_narrow_trees(n_nodes, shape):
+    """The HBM-bound regime of the benchmark: deep, narrow trees of one (16 nodes) and two (24 nodes) row tiles,
+    in the launch configuration the library picks for them."""
+    w = _build(n_nodes, shape)
+    st = sage.new_status()
+    out = sage.sage_tree_attention(w["q"], w["k"], w["v"], w["page_table"], w["seq_len"], w["parent"], w["offs"],
+                                   1.0 / np.sqrt(D), status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0, sage.status_string(int(st.item()))
+    assert bool(torch.isfinite(out.float()).all())
+    offs = np.array([0, n_nodes], np.int32)
     for layer in SAMPLED_LAYERS:
         want = oracle.tree_attention(host_bits(w["q"][layer]), host_bits(w["k"][layer]), host_bits(w["v"][layer]),
                                      w["perm"].reshape(1, -1), np.array([L], np.int32), w["tree"]["parent"], offs,
