@@ -255,11 +255,14 @@ const char *sage_status_string(int code);
  * to run the time-out path without faulting or hanging the device; leave it alone otherwise. */
 void sage_debug_attention_waits(long long wait_cycles, int producer_off);
 
-/* sage_tree_attention has two schedules and picks one per launch: a streaming one (one resident thread
- * block per multiprocessor walks an equal share of all the work) for long, HBM-bound launches, and a
- * split one (a grid over context slices, row pairs and KV heads, plus a merge) for tensor-bound trees
- * and short launches.  schedule = 1 forces the streaming one, 2 the split one, anything else restores
- * the automatic choice.  For tests and measurements (no counterpart in the paper). */
+/* sage_tree_attention picks a schedule per launch: a streaming one (one resident thread block per
+ * multiprocessor walks an equal share of all the work in steps of 128 keys; trees of up to 128 query
+ * rows per KV head alternate their steps between two accumulator slots, trees of up to 256 keep two row
+ * tiles per block) for long, HBM-bound launches, and a split one (a grid over context slices, row pairs
+ * and KV heads, plus a merge) for tensor-bound trees and short launches.  schedule = 1 forces the
+ * streaming one, 2 the split one, 3 the streaming one on two-block clusters that share every K/V tile
+ * (one tensor-core instruction stream per cluster; measured slower, kept for comparison), anything
+ * else restores the automatic choice.  For tests and measurements (no counterpart in the paper). */
 void sage_debug_attention_schedule(int schedule);
 
 #ifdef __cplusplus

@@ -294,7 +294,7 @@ def sage_debug_attention_waits(wait_cycles: int = 0, producer_off: bool = False)
 
 
 def sage_debug_attention_schedule(schedule: int = 0) -> None:
-    """0: the library picks the attention schedule per launch; 1: streaming; 2: split."""
+    """0: the library picks the attention schedule per launch; 1: streaming; 2: split; 3: streaming on two-block clusters."""
     _lib.sage_debug_attention_schedule(int(schedule))
 
 

@@ -1,31 +1,42 @@
 // Tree-masked verification attention over a paged bf16 KV cache (Section 2.2;
-// Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2), sm_100a.
+// Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2), sm_100a:
+// the C entry points, the choice of schedule, and the streaming kernel for trees of one
+// row tile.  tree_attention_rows.cu holds the streaming kernel for two row tiles per CTA,
+// tree_attention_split.cu the split schedule.
 //
 // Work decomposition.  The N tree nodes x G query heads that share one KV head form
-// M = N*G query rows (<= 512).  An *item* is one (layer, sequence, KV head); its work
-// is measured in steps of 128 keys (two 64-token pages).  All items are laid end to
-// end and cut into equal ranges of steps, one range per *gang*; a gang is the 1 or 2
-// CTAs (one per 256 query rows) that walk the same range side by side, so that the
-// second CTA finds the K/V of the first in L2.  A kernel launch is one resident CTA
-// per SM that loops over the segments of its range: whole items write their output
-// directly, items cut by a range boundary leave unnormalised partial results that
-// attention_merge_kernel combines.  Nothing waits on another CTA.
+// M = N*G query rows; here M <= 128, one row tile (the pair form takes more: see below).
+// An *item* is one (layer, sequence, KV head); its work is measured in steps of 128 keys
+// (two 64-token pages).  All items are laid end to end and cut into equal ranges of steps,
+// one range per *gang* (one CTA; in the pair form the CTA pairs that cover a tree's row
+// tiles).  A kernel launch is one resident CTA per SM that loops over the segments of its
+// range: whole items write their output directly, items cut by a range boundary leave
+// unnormalised partial results that attention_merge_kernel combines.  No CTA waits on
+// another one outside its pair.
 //
-// Inside a CTA (384 threads), per 128-key step and 128-row tile t:
+// Inside a CTA (384 threads): tensor memory holds two slots t of (S_t 128 x 128 fp32 scores,
+// O_t 128 x 128 fp32 accumulator).  Both slots work for the same 128 query rows: slot t takes
+// the steps s0 + t, s0 + t + 2, ... of a segment, so that the softmax of one step runs while
+// the tensor pipe works on the next step (with one slot the chain scores -> softmax -> P V of
+// a row tile is strictly serial); the two accumulators are combined in the epilogue.
 //   TMA      : K and V tiles (2 pages x 2 d-halves) -> 128B-swizzled shared memory, rings of
-//              3 K tiles and 2 V tiles, mbarriers; the two query tiles also arrive by TMA
-//   tcgen05  : S_t = Q_t K^T (128 x 128, fp32) into TMEM; one warp issues for both row tiles, through
-//              one elected lane, with warp-uniform descriptor arithmetic
-//   softmax  : one warpgroup per row tile, one thread per row: tcgen05.ld S in four 32-column
+//              3 K tiles and 3 V tiles, mbarriers; the query tile also arrives by TMA
+//   tcgen05  : S_t = Q K^T into TMEM; one thread issues for both slots, in blocks
+//              [P V of step i-2, scores of step i]
+//   softmax  : one warpgroup per slot, one thread per row: tcgen05.ld S in four 32-column
 //              chunks, online softmax in fp32 (log2 domain, lazy rescale), P -> bf16 back
 //              into TMEM over the first 64 columns of S_t
 //   tcgen05  : O_t += P_t V with P as the TMEM A operand, V MN-major from shared memory
 // A 128 x 64 score MMA occupies the tensor pipe exactly as long as a 128 x 128 one (64 clocks
-// per K=16 slice, measured), hence the 128-key step.  The two row tiles alternate on the
-// tensor pipe: while one tile's warpgroup runs its softmax, the pipe works on the other tile.
+// per K=16 slice, measured), hence the 128-key step.
 // TMEM map (512 columns): S_t [128t, 128t+128), O_t [256+128t, 384+128t).
-// All waits are bounded: on expiry the CTA records SAGE_STATUS_TIMEOUT, waits (bounded) for
-// its copies and MMAs in flight, frees its TMEM and returns.
+//
+// Pair form (tree_attention_kernel<true>, forced for measurements only): clusters of two CTAs
+// with one MMA stream (cta_group::2, M = 256), one row tile per CTA; each CTA holds half of every
+// K tile and half of every V tile, so a step's K and V enter the pair's shared memory once.
+//
+// All waits are bounded: on expiry the CTA (both CTAs of a pair) records SAGE_STATUS_TIMEOUT,
+// waits (bounded) for its copies and MMAs in flight, frees its TMEM and returns.
 #include <cuda.h>
 
 #include <mutex>
