@@ -246,6 +246,27 @@ def test_tree_attention_edges(L, N, G, schedule):
     check_attention(got[0], oracle_attention_layer(c, 0), bf16_slack=True)
 
 
+@pytest.mark.parametrize("G,Ns,Ls", [(8, [1, 3, 2, 4, 6], [0, 130, 64, 700, 257]),
+                                     (1, [10, 20, 34], [500, 0, 129]),
+                                     (4, [8, 8, 8, 8], [127, 128, 129, 1])])
+def test_tree_attention_batches_of_small_trees_stacked_layers(G, Ns, Ls, schedule):
+    """Trees of one row tile (N * G <= 128 query rows per KV head) in ragged batches over three stacked
+    layers: the shape of the alternating-slot streaming kernel.  The sequences are short, so most ranges of
+    steps cut an item (partial results and the merge), and segments of one, two and three steps all occur
+    (a slot without steps, slots of unequal length)."""
+    r = rng(7000 + G)
+    Hkv, n_layers = 2, 3
+    trees = [random_tree(r, n) for n in Ns]
+    kv = make_kv_cache(r, Ls, Ns, [l // 2 for l in Ls], Hkv, n_layers=n_layers, shuffle=True, spare_frac=0.3)
+    c = {"q": make_q(r, sum(Ns), Hkv * G, n_layers=n_layers), **kv,
+         "parent": np.concatenate([t["parent"] for t in trees]).astype(np.int32),
+         "node_offsets": np.concatenate([[0], np.cumsum(Ns)]).astype(np.int32),
+         "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.11}
+    got = gpu_attention(c)
+    for layer in range(n_layers):
+        check_attention(got[layer], oracle_attention_layer(c, layer), bf16_slack=True)
+
+
 def test_tree_attention_chain_and_star_trees(schedule):
     r = rng(9)
     for tree in (chain_tree(40), star_tree(50)):
