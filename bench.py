@@ -640,7 +640,12 @@ def run_cuda(args):
                          "bound": "hbm", "achieved": r24["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": r24["frac_hbm"], "traffic": None, "ms_per_launch": r24["ms_per_launch"],
                          "algorithmic_bytes": r24["algorithmic_bytes"], "target_frac": 0.70,
-                         "target_met": bool(r24["frac_hbm"] >= 0.70), "peak_source": peaks["source"] + " (copy bandwidth)"}
+                         "target_met": bool(r24["frac_hbm"] >= 0.70), "peak_source": peaks["source"] + " (copy bandwidth)",
+                         "one_row_tile": {"kernel": f"tree_attention, 16-node (8,2) tree (128 query rows per KV head), "
+                                                    f"{N_LAYERS} stacked layers, 16k context",
+                                          "achieved": by_tree[0]["gbs"], "frac": by_tree[0]["frac_hbm"],
+                                          "ms_per_launch": by_tree[0]["ms_per_launch"],
+                                          "target_met": bool(by_tree[0]["frac_hbm"] >= 0.70)}}
         logits_bytes = float(N_NODES) * V * 4
         line = {
             "metric": "tree-verify rounds/s", "value": value, "unit": "rounds/s", "n_gpus": world, "steps": steps,
