@@ -621,9 +621,11 @@ def run_cuda(args):
                             "sample": f"{sample_s:.1f} s of oracle work: the whole logits side (60 draft + 60 target "
                                       f"rows), attention, acceptance and compaction of 1 of the {N_LAYERS} layers; "
                                       "the other layers are extrapolated"}
-        # expand (3), select + hand-over (2), attention (1: at this shape the split schedule runs with one context
-        # slice per CTA, so no merge kernel is launched), target top-1 (2), accept (1), compact + advance (2)
-        launches = 3 + 2 + 1 + 2 + 1 + 2
+        # expand (3), select + hand-over (2), attention (5: the library starts the kernels for trees of one row
+        # tile (+ merge), two row tiles (+ merge) and more, and the tree size found on the device leaves the last
+        # one running; at this shape it has one context slice per CTA, so no merge of its own), target top-1 (2),
+        # accept (1), compact + advance (2).  With --layers below 9 the launch is short and only one kernel starts.
+        launches = 3 + 2 + 5 + 2 + 1 + 2
         # Which tensor peak applies: the burst figure when the SM clock stayed at its maximum through the
         # timed region, the sustained one when the power cap pulled it down.  Both fractions are printed.
         sm, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")

@@ -206,10 +206,14 @@ int sage_build_ancestor_mask(const int32_t *parent, const int32_t *node_offsets,
  * q, out: bf16 [n_layers][sum_nodes][n_q_heads][head_dim]; `sum_nodes` is the node
  * capacity of those buffers (>= node_offsets[batch]).  Softmax and accumulation in
  * fp32.  Rows of the cache beyond L_b+N_b may hold anything (NaN included).
- * ws: sage_tree_attention_workspace_size(...) bytes (a fixed amount per streaming multiprocessor of
- * the current device, independent of the problem size: the kernel is one resident thread block
- * per multiprocessor, and each keeps at most two partial results for sequences that a work
- * boundary cuts). */
+ * Rows of q and out beyond node_offsets[batch] are neither read nor written.  The work is scheduled from
+ * the trees actually present, not from the capacity: where the host cannot tell which of the library's
+ * kernels suits them (a long launch whose capacity allows trees of more than 128 query rows per KV
+ * head), every candidate is started, each finds the largest tree of the batch in node_offsets on the
+ * device, and all but the right one leave at once.
+ * ws: sage_tree_attention_workspace_size(...) bytes: partial results of the sequences that a work
+ * boundary or a context slice cuts (the larger of a fixed amount per streaming multiprocessor and an
+ * amount per layer, context slice and query row). */
 int sage_tree_attention(const void *q, const void *k_pool, const void *v_pool,
                         int64_t layer_stride_elems, int n_layers, int n_pages,
                         const int32_t *page_table, int max_pages_per_seq, const int32_t *seq_len,

@@ -86,6 +86,7 @@ struct AttnParams {
     float scale_log2;          // sm_scale * log2(e)
     long long wait_cycles;     // budget of every on-device wait
     int producer_off;          // diagnostics: the TMA warp issues no copies (every consumer wait then runs out)
+    int select;                // which tree sizes this launch is for (schedule_selected)
 };
 
 struct __align__(16) Shared {
@@ -554,7 +555,8 @@ tree_attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap qm
     // ---- this gang's range of steps (warp 0 computes, everybody reads)
     if (warp == 0) {
         int err = 0;
-        const int Wb = steps_per_head(p, lane, &err);
+        const bool mine = schedule_selected(p.select, max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane));
+        const int Wb = mine ? steps_per_head(p, lane, &err) : 0;
         if (err) report_status(p.status, err);
         const long long W = (long long)p.n_layers * p.Hkv * Wb;
         long long begin = 0, end = 0;
@@ -1089,7 +1091,8 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(AttnParams p) {
     const int k_cut = blockIdx.x + 1;                   // boundary between gang k_cut - 1 and gang k_cut
     if (warp == 0) {
         int err = 0, b = 0, s0 = 0;
-        const int Wb = steps_per_head(p, lane, &err);
+        const bool mine = schedule_selected(p.select, max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane));
+        const int Wb = mine ? steps_per_head(p, lane, &err) : 0;
         if (Wb > 0) {
             const long long W = (long long)p.n_layers * p.Hkv * Wb;
             const int n_act = active_gangs(W, p.n_gangs);
@@ -1267,13 +1270,13 @@ size_t workspace_size(int n_layers, int batch, int sum_nodes, int n_q_heads, int
 int launch(const void* q, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
            const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
            int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
-           int producer_off, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream);
+           int producer_off, int select, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream);
 }  // namespace split
 
 // The streaming schedule for trees of more than one row tile (tree_attention_rows.cu).
 namespace rows {
 size_t workspace_size(int n_ctas);
-int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+int launch(int n_ctas, int select, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
            const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
            int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
            int producer_off, const CUtensorMap& qmap, const CUtensorMap& kmap, const CUtensorMap& vmap,
@@ -1282,24 +1285,28 @@ int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int
 
 // Which schedule runs a launch.
 //   streaming: persistent CTAs that walk equal ranges of 128-key steps.  One row tile (up to 128 query rows
-//     per KV head): the kernel of this file, single form, which is HBM-bound.  More: two row tiles per CTA
-//     (tree_attention_rows.cu); chosen up to 256 rows, where one CTA holds the whole tree and nothing is read twice.
+//     per KV head): the kernel of this file, single form, which is HBM-bound.  Two row tiles (up to 256 rows):
+//     two row tiles per CTA (tree_attention_rows.cu): one CTA holds the whole tree and nothing is read twice.
 //   split: grid over (context slice, row pair, layer x sequence x KV head), 64-key steps: wins where the
 //     work is tensor-bound (more than 256 rows) and where a launch is too short to give every SM a long
 //     stream (single layers, short contexts: fixed costs dominate).
 //   pairs: the kernel of this file in its pair form; measured slower than the others everywhere (the
 //     hand-overs between the two CTAs lengthen the per-step dependency chain), so never chosen, only forced.
-enum Schedule { kAlternating, kRows, kSplit, kPairs };
+// The host knows how long a launch is, but of the trees only an upper bound: sum_nodes is the size of the
+// caller's node arrays, and a decode loop that lives on the device keeps arrays of full capacity whatever
+// the trees of a round look like.  So a long launch whose bound allows more than one row tile starts every
+// streaming or split kernel that might apply, each told which tree sizes are its own; each works the largest
+// tree of the batch out from node_offsets and all but one leave at once (a few microseconds in all).
+enum Schedule { kAlternating, kRows, kSplit, kPairs, kOnDevice };
 constexpr int kStreamMinSteps = 16;
 static Schedule pick_schedule(int n_layers, int batch, int sum_nodes, int n_kv_heads, int G, int max_pages_per_seq) {
     const int tiles = row_tiles(sum_nodes, G);
     if (g_schedule == 1) return tiles == 1 ? kAlternating : kRows;
     if (g_schedule == 2) return kSplit;
     if (g_schedule == 3) return tiles == 1 ? kAlternating : kPairs;
-    if (tiles > 2) return kSplit;
     const long long steps = (long long)n_layers * batch * n_kv_heads * ((max_pages_per_seq + 1) / 2);   // upper bound
     if (steps < (long long)kStreamMinSteps * resident_ctas()) return kSplit;
-    return tiles == 1 ? kAlternating : kRows;
+    return tiles == 1 ? kAlternating : kOnDevice;
 }
 
 }  // namespace sage
@@ -1361,16 +1368,30 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     if (sched == kSplit)
         return split::launch(q, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent, node_offsets, batch,
                              sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status, g_wait_cycles, g_producer_off,
-                             kmap, vmap, as_stream(stream));
+                             0, kmap, vmap, as_stream(stream));
     if (!make_q_map(&qmap, q, n_layers, sum_nodes, n_kv_heads, G)) return SAGE_ERR_CUDA;
     if (sched == kRows)
-        return rows::launch(resident_ctas(), n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent,
+        return rows::launch(resident_ctas(), 0, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent,
                             node_offsets, batch, sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status,
                             g_wait_cycles, g_producer_off, qmap, kmap, vmap, as_stream(stream));
+    const int tiles = row_tiles(sum_nodes, G);
+    if (sched == kOnDevice) {
+        // the kernels for two row tiles and (if the bound allows them) for more; the one for one row tile follows below
+        int rc = rows::launch(resident_ctas(), 2, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent,
+                              node_offsets, batch, sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status,
+                              g_wait_cycles, g_producer_off, qmap, kmap, vmap, as_stream(stream));
+        if (rc != SAGE_OK) return rc;
+        if (tiles > 2) {
+            if ((long long)n_layers * batch * n_kv_heads > 65535) return SAGE_ERR_UNSUPPORTED;    // grid limit of the split schedule
+            rc = split::launch(q, n_layers, n_pages, page_table, max_pages_per_seq, seq_len, parent, node_offsets, batch,
+                               sum_nodes, n_q_heads, n_kv_heads, sm_scale, out, ws, status, g_wait_cycles,
+                               g_producer_off, 3, kmap, vmap, as_stream(stream));
+            if (rc != SAGE_OK) return rc;
+        }
+    }
     const int n_ctas = resident_ctas();
     AttnParams p{};
     // one row tile: single CTAs; more (pair form only): CTA pairs, two row tiles each
-    const int tiles = row_tiles(sum_nodes, G);
     const bool pair = sched == kPairs;
     p.n_rp = pair ? 2 * ((tiles + 1) / 2) : 1;
     p.n_gangs = n_ctas / p.n_rp;
@@ -1384,6 +1405,7 @@ extern "C" int sage_tree_attention(const void* q, const void* k_pool, const void
     p.scale_log2 = sm_scale * 1.4426950408889634f;
     p.wait_cycles = g_wait_cycles;
     p.producer_off = g_producer_off;
+    p.select = sched == kOnDevice ? 1 : 0;
 
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static bool attr_set[64] = {};

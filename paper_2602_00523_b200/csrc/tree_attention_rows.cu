@@ -59,7 +59,8 @@ struct AttnParams {
     int32_t* status;
     int n_layers, batch, sum_nodes, n_pages, max_pages;
     int Hq, Hkv, G;
-    int n_gangs, n_rp;         // gangs in the launch, CTAs per gang (row pairs of the largest possible tree)
+    int n_ctas, n_rp;          // CTAs of the launch; most CTAs a gang can have (row pairs of the largest possible tree)
+    int select;                // which tree sizes this launch is for (schedule_selected)
     float scale_log2;          // sm_scale * log2(e)
     long long wait_cycles;     // budget of every on-device wait
     int producer_off;          // diagnostics: the TMA warp issues no copies (every consumer wait then runs out)
@@ -76,6 +77,7 @@ struct __align__(16) Shared {
     uint64_t drain;            // abort path: everything issued so far has retired
     long long range_begin, range_end;
     int first_lg, first_b, first_s0;
+    int n_rp, n_gangs;         // CTAs per gang (row pairs of the largest tree of this batch) and gangs, found on the device
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -481,18 +483,24 @@ tree_attention_rows_kernel(const AttnParams p, const __grid_constant__ CUtensorM
     Shared* sh = reinterpret_cast<Shared*>(sV + kVStages * kTileBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int member = blockIdx.x % p.n_rp, gang = blockIdx.x / p.n_rp;
 
-    // ---- this gang's range of steps (warp 0 computes, everybody reads)
+    // ---- the gangs of this launch and this gang's range of steps (warp 0 computes, everybody reads).
+    // A gang has as many CTAs as the largest tree of the batch has row pairs, which only the device knows
+    // when the caller's node arrays are larger than the trees in them.
     if (warp == 0) {
         int err = 0;
-        const int Wb = steps_per_head(p, lane, &err);
+        const int rows_max = max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane);
+        const bool mine = schedule_selected(p.select, rows_max);
+        const int n_rp = min(p.n_rp, max(1, (rows_max + kRowsPerCta - 1) / kRowsPerCta));
+        const int n_gangs = p.n_ctas / n_rp;
+        const int gang = blockIdx.x / n_rp;
+        const int Wb = mine ? steps_per_head(p, lane, &err) : 0;
         if (err) report_status(p.status, err);
         const long long W = (long long)p.n_layers * p.Hkv * Wb;
         long long begin = 0, end = 0;
         int lg = 0, b = 0, s0 = 0;
         if (W > 0) {
-            const int n_act = active_gangs(W, p.n_gangs);
+            const int n_act = active_gangs(W, n_gangs);
             if (gang < n_act) {
                 begin = gang_begin(W, n_act, gang);
                 end = gang_begin(W, n_act, gang + 1);
@@ -505,10 +513,13 @@ tree_attention_rows_kernel(const AttnParams p, const __grid_constant__ CUtensorM
         if (lane == 0) {
             sh->range_begin = begin; sh->range_end = end;
             sh->first_lg = lg; sh->first_b = b; sh->first_s0 = s0;
+            sh->n_rp = n_rp; sh->n_gangs = n_gangs;
         }
     }
     __syncthreads();
     if (sh->range_end <= sh->range_begin) return;       // uniform: nothing to do, nothing allocated yet
+    const int n_rp = sh->n_rp;
+    const int member = blockIdx.x % n_rp, gang = blockIdx.x / n_rp;
 
     // ---- set-up: barriers, TMEM
     if (tid == 0) {
@@ -818,7 +829,7 @@ tree_attention_rows_kernel(const AttnParams p, const __grid_constant__ CUtensorM
                 const size_t row = (size_t)(sg.n0 + node) * p.Hq + sg.g * p.G + (row_ok ? R % p.G : 0);
                 oo = p.out + ((size_t)sg.layer * p.sum_nodes * p.Hq + row) * kHeadDim;
             } else {
-                const size_t pr = (((size_t)gang * 2 + (sg.at_range_begin ? 0 : 1)) * p.n_rp + member) * kRowsPerCta +
+                const size_t pr = (((size_t)gang * 2 + (sg.at_range_begin ? 0 : 1)) * n_rp + member) * kRowsPerCta +
                                   t * kRowTile + r;
                 po = p.part_o + pr * kHeadDim;
                 if (row_ok) { p.part_ml[pr * 2] = m_ref; p.part_ml[pr * 2 + 1] = l_sum; }
@@ -868,24 +879,29 @@ tree_attention_rows_kernel(const AttnParams p, const __grid_constant__ CUtensorM
 // item's segments: which gangs hold them, and in which of their two partial slots, follows from
 // the positions alone.
 __global__ void __launch_bounds__(256) attention_rows_merge_kernel(AttnParams p) {
-    __shared__ int s_Wb, s_b, s_s0;
+    __shared__ int s_Wb, s_b, s_s0, s_n_rp;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_cut = blockIdx.x + 1;                   // boundary between gang k_cut - 1 and gang k_cut
     if (warp == 0) {
         int err = 0, b = 0, s0 = 0;
-        const int Wb = steps_per_head(p, lane, &err);
+        // the same gang layout as the attention kernel worked out
+        const int rows_max = max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane);
+        const bool mine = schedule_selected(p.select, rows_max);
+        const int n_rp = min(p.n_rp, max(1, (rows_max + kRowsPerCta - 1) / kRowsPerCta));
+        const int Wb = mine ? steps_per_head(p, lane, &err) : 0;
         if (Wb > 0) {
             const long long W = (long long)p.n_layers * p.Hkv * Wb;
-            const int n_act = active_gangs(W, p.n_gangs);
+            const int n_act = active_gangs(W, p.n_ctas / n_rp);
             if (k_cut < n_act) locate(p, lane, (int)(gang_begin(W, n_act, k_cut) % Wb), &b, &s0);
         }
-        if (lane == 0) { s_Wb = Wb; s_b = b; s_s0 = s0; }
+        if (lane == 0) { s_Wb = Wb; s_b = b; s_s0 = s0; s_n_rp = n_rp; }
     }
     __syncthreads();
     const int Wb = s_Wb;
     if (Wb <= 0) return;
+    const int n_rp = s_n_rp;
     const long long W = (long long)p.n_layers * p.Hkv * Wb;
-    const int n_act = active_gangs(W, p.n_gangs);
+    const int n_act = active_gangs(W, p.n_ctas / n_rp);
     if (k_cut >= n_act || s_s0 == 0) return;            // no such boundary, or it falls between two items
     const long long cut = gang_begin(W, n_act, k_cut);
     const int lg = (int)(cut / Wb), b = s_b;
@@ -903,7 +919,7 @@ __global__ void __launch_bounds__(256) attention_rows_merge_kernel(AttnParams p)
         const int member = R / kRowsPerCta, Rl = R % kRowsPerCta;
         auto slot_row = [&](int k) -> size_t {
             const int slot = (k == k_first && first_mid_range) ? 1 : 0;
-            return (((size_t)k * 2 + slot) * p.n_rp + member) * kRowsPerCta + Rl;
+            return (((size_t)k * 2 + slot) * n_rp + member) * kRowsPerCta + Rl;
         };
         float mx = -INFINITY;
         for (int k = k_first + lane; k <= k_last; k += 32) {
@@ -941,7 +957,7 @@ static int row_pairs(int sum_nodes, int G) {
 // Two partial slots (head and tail of its range) per resident CTA, independent of the problem size.
 size_t workspace_size(int n_ctas) { return (size_t)n_ctas * 2 * kRowsPerCta * (kHeadDim + 2) * sizeof(float); }
 
-int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+int launch(int n_ctas, int select, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
            const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
            int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
            int producer_off, const CUtensorMap& qmap, const CUtensorMap& kmap, const CUtensorMap& vmap,
@@ -949,7 +965,8 @@ int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int
     const int G = n_q_heads / n_kv_heads;
     AttnParams p{};
     p.n_rp = row_pairs(sum_nodes, G);
-    p.n_gangs = n_ctas / p.n_rp;
+    p.n_ctas = (n_ctas / p.n_rp) * p.n_rp;          // whole gangs whatever the gang size turns out to be (1 or 2)
+    p.select = select;
     p.out = (__nv_bfloat16*)out;
     p.part_o = (float*)ws;
     p.part_ml = (float*)ws + (size_t)n_ctas * 2 * kRowsPerCta * kHeadDim;
@@ -970,9 +987,10 @@ int launch(int n_ctas, int n_layers, int n_pages, const int32_t* page_table, int
             return SAGE_ERR_CUDA;
         attr_set[dev] = true;
     }
-    tree_attention_rows_kernel<<<p.n_gangs * p.n_rp, kAttnThreads, kSmemBytes, stream>>>(p, qmap, kmap, vmap);
-    if (p.n_gangs > 1) {
-        dim3 mg((unsigned)(p.n_gangs - 1), (unsigned)((p.n_rp * kRowsPerCta + 31) / 32));
+    tree_attention_rows_kernel<<<p.n_ctas, kAttnThreads, kSmemBytes, stream>>>(p, qmap, kmap, vmap);
+    if (p.n_ctas > 1) {
+        // one block per possible boundary between two gangs' ranges and 32-row chunk; those that find no cut item leave
+        dim3 mg((unsigned)(p.n_ctas - 1), (unsigned)((p.n_rp * kRowsPerCta + 31) / 32));
         attention_rows_merge_kernel<<<mg, 256, 0, stream>>>(p);
     }
     return launch_status();

@@ -52,6 +52,7 @@ struct AttnParams {
     float scale_log2;  // sm_scale * log2(e)
     long long wait_cycles;     // budget of every on-device wait
     int producer_off;          // diagnostics: the TMA warp issues no copies (every consumer wait then runs out)
+    int select;                // which tree sizes this launch is for (schedule_selected)
 };
 
 struct __align__(8) Barriers {
@@ -318,6 +319,8 @@ tree_attention_split_kernel(const AttnParams p, const __grid_constant__ CUtensor
     const int layer = blockIdx.z / (p.Hkv * p.batch);
 
     // ---- uniform early exits (before any barrier or TMEM is touched)
+    // (every warp works the batch's largest tree out for itself: the same answer everywhere, no barrier)
+    if (p.select != 0 && !schedule_selected(p.select, max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane))) return;
     const int n0 = p.node_offsets[b];
     const int N = p.node_offsets[b + 1] - n0;
     const int L = p.seq_len[b];
@@ -695,6 +698,7 @@ __global__ void attention_split_merge_kernel(AttnParams p) {
     const size_t row = (size_t)blockIdx.x * warps + (threadIdx.x >> 5);
     const int layer = blockIdx.y;
     const int lane = threadIdx.x & 31;
+    if (p.select != 0 && !schedule_selected(p.select, max_tree_rows(p.node_offsets, p.batch, p.sum_nodes, p.G, lane))) return;
     if (row >= rows_total) return;
     const int node = (int)(row / p.Hq);
     if (node >= p.node_offsets[p.batch]) return;       // rows past the live nodes were never written
@@ -759,7 +763,7 @@ size_t workspace_size(int n_layers, int batch, int sum_nodes, int n_q_heads, int
 int launch(const void* q, int n_layers, int n_pages, const int32_t* page_table, int max_pages_per_seq,
            const int32_t* seq_len, const int32_t* parent, const int32_t* node_offsets, int batch, int sum_nodes,
            int n_q_heads, int n_kv_heads, float sm_scale, void* out, void* ws, int32_t* status, long long wait_cycles,
-           int producer_off, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream) {
+           int producer_off, int select, const CUtensorMap& kmap, const CUtensorMap& vmap, cudaStream_t stream) {
     const int G = n_q_heads / n_kv_heads;
     const int S = pick_splits(n_layers, batch, n_kv_heads, G, max_pages_per_seq, sum_nodes);
     AttnParams p{};
@@ -774,6 +778,7 @@ int launch(const void* q, int n_layers, int n_pages, const int32_t* page_table, 
     p.scale_log2 = sm_scale * 1.4426950408889634f;
     p.wait_cycles = wait_cycles;
     p.producer_off = producer_off;
+    p.select = select;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static bool attr_set[64] = {};
     int dev = 0;

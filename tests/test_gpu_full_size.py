@@ -81,6 +81,35 @@ def test_attention_80_layers_deep_narrow_trees(n_nodes, shape):
         check_attention(host_bits(out[layer]), want)
 
 
+@pytest.mark.parametrize("n_nodes,shape", [(9, (8, 1)), (24, (8, 2)), (60, (3, 10))], ids=["9_nodes", "24_nodes", "60_nodes"])
+def test_attention_80_layers_node_arrays_of_full_capacity(n_nodes, shape):
+    """A decode loop that lives on the device keeps node arrays of full capacity (64 nodes) whatever the
+    tree of a round looks like, so the host only knows an upper bound of the tree size: the library then
+    starts every kernel that might apply and the tree size found on the device (node_offsets) picks the one
+    that runs.  The rows past the tree must stay untouched."""
+    cap = sage.SAGE_MAX_NODES
+    w = _build(n_nodes, shape)
+    dev = w["q"].device
+    q = torch.zeros((N_LAYERS, cap, HQ, D), dtype=torch.bfloat16, device=dev)
+    q[:, :n_nodes] = w["q"]
+    parent = np.full(cap, -1, np.int32)
+    parent[:n_nodes] = w["tree"]["parent"]
+    out = torch.full_like(q, 7.0)
+    st = sage.new_status()
+    sage.sage_tree_attention(q, w["k"], w["v"], w["page_table"], w["seq_len"], dev_i32(parent), w["offs"],
+                             1.0 / np.sqrt(D), out=out, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0, sage.status_string(int(st.item()))
+    assert bool((out[:, n_nodes:].float() == 7.0).all())
+    assert bool(torch.isfinite(out[:, :n_nodes].float()).all())
+    offs = np.array([0, n_nodes], np.int32)
+    for layer in (SAMPLED_LAYERS[0], SAMPLED_LAYERS[-1]):
+        want = oracle.tree_attention(host_bits(q[layer, :n_nodes]), host_bits(w["k"][layer]), host_bits(w["v"][layer]),
+                                     w["perm"].reshape(1, -1), np.array([L], np.int32), w["tree"]["parent"], offs,
+                                     HQ, HKV, D, P, 1.0 / np.sqrt(D))
+        check_attention(host_bits(out[layer, :n_nodes]), want)
+
+
 def test_compaction_80_layers_moves_exactly_the_accepted_rows():
     w = _build()
     k0, v0 = w["k"].clone(), w["v"].clone()
