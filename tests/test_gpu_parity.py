@@ -199,11 +199,12 @@ def test_select_tree_edges_and_handover():
 
 
 # ------------------------------------------------------------------ attention
-@pytest.fixture(params=[1, 2, 3], ids=["streaming", "split", "pairs"])
+@pytest.fixture(params=[0, 1, 2, 3], ids=["auto", "streaming", "split", "pairs"])
 def schedule(request):
-    """sage_tree_attention picks a schedule per launch; the parity tests force each in turn (streaming: persistent
-    thread blocks, one or two row tiles each; split: grid over context slices; pairs: streaming with two-block
-    clusters that share every K/V tile)."""
+    """sage_tree_attention picks a schedule per launch (auto: from the launch's length on the host and from
+    the trees on the device); the parity tests also force each in turn (streaming: persistent thread blocks,
+    one or two row tiles each; split: grid over context slices; pairs: streaming with two-block clusters that
+    share every K/V tile)."""
     sage.sage_debug_attention_schedule(request.param)
     yield request.param
     sage.sage_debug_attention_schedule(0)
