@@ -268,6 +268,25 @@ def test_tree_attention_batches_of_small_trees_stacked_layers(G, Ns, Ls, schedul
         check_attention(got[layer], oracle_attention_layer(c, layer), bf16_slack=True)
 
 
+@pytest.mark.parametrize("Ns,kernel", [([5, 12, 9], "one row tile"), ([5, 30, 9], "two row tiles"), ([5, 40, 9], "split")])
+def test_tree_attention_long_launch_picks_its_kernel_from_the_largest_tree_of_the_batch(Ns, kernel):
+    """A launch long enough for the streaming schedule (26 stacked layers of three 2000-token sequences),
+    whose node arrays allow more row tiles than the trees use: the library starts every kernel that might
+    apply and the largest tree of the batch, found on the device, decides which one runs."""
+    r = rng(8100 + Ns[1])
+    Hkv, G, n_layers = 2, 8, 26
+    Ls = [2000, 1990, 2040]
+    trees = [random_tree(r, n) for n in Ns]
+    kv = make_kv_cache(r, Ls, Ns, [l // 2 for l in Ls], Hkv, n_layers=n_layers, shuffle=True, spare_frac=0.2)
+    c = {"q": make_q(r, sum(Ns), Hkv * G, n_layers=n_layers), **kv,
+         "parent": np.concatenate([t["parent"] for t in trees]).astype(np.int32),
+         "node_offsets": np.concatenate([[0], np.cumsum(Ns)]).astype(np.int32),
+         "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.0884}
+    got = gpu_attention(c)
+    for layer in (0, 11, n_layers - 1):
+        check_attention(got[layer], oracle_attention_layer(c, layer))
+
+
 def test_tree_attention_chain_and_star_trees(schedule):
     r = rng(9)
     for tree in (chain_tree(40), star_tree(50)):
