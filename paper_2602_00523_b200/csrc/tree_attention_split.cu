@@ -2,7 +2,8 @@
 // Algorithm 1, the target pass over all tree tokens; Section 3.3 Phase 2), sm_100a:
 // the split schedule, used for launches that are tensor-bound (more than 256 query rows
 // per KV head) or too small to give every SM a long stream of work (single layers,
-// short contexts).  tree_attention.cu holds the streaming schedule and the dispatch.
+// short contexts).  tree_attention.cu holds the dispatch and, with tree_attention_rows.cu, the
+// streaming schedule.
 //
 // Flash-decoding layout.  The N tree nodes x G query heads that share one KV head
 // form M = N*G query rows (<= 512).  A CTA owns up to two 128-row tiles of them and
