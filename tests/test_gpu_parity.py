@@ -287,6 +287,28 @@ def test_tree_attention_long_launch_picks_its_kernel_from_the_largest_tree_of_th
         check_attention(got[layer], oracle_attention_layer(c, layer))
 
 
+@pytest.mark.parametrize("G", [2, 8])
+def test_tree_attention_batch_of_forty_sequences(G, schedule):
+    """More sequences than a warp has lanes (the schedules walk the batch 32 sequences at a time), with
+    contexts from empty to a few steps and trees of one to three nodes; two stacked layers."""
+    r = rng(9100 + G)
+    Hkv, n_layers, B = 2, 2, 40
+    Ns = [int(x) for x in r.integers(1, 4, size=B)]
+    if G == 2:
+        Ns = [1] * B
+    Ls = [int(x) for x in r.integers(0, 400, size=B)]
+    Ls[0], Ls[33], Ls[39] = 0, 128, 127
+    trees = [random_tree(r, n) for n in Ns]
+    kv = make_kv_cache(r, Ls, Ns, [l // 2 for l in Ls], Hkv, n_layers=n_layers, shuffle=True, spare_frac=0.25)
+    c = {"q": make_q(r, sum(Ns), Hkv * G, n_layers=n_layers), **kv,
+         "parent": np.concatenate([t["parent"] for t in trees]).astype(np.int32),
+         "node_offsets": np.concatenate([[0], np.cumsum(Ns)]).astype(np.int32),
+         "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.1}
+    got = gpu_attention(c)
+    for layer in range(n_layers):
+        check_attention(got[layer], oracle_attention_layer(c, layer), bf16_slack=True)
+
+
 def test_tree_attention_chain_and_star_trees(schedule):
     r = rng(9)
     for tree in (chain_tree(40), star_tree(50)):
