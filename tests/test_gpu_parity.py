@@ -355,6 +355,38 @@ def test_tree_attention_wait_that_runs_out_reports_timeout_and_leaves_the_contex
     check_attention(gpu_attention(c)[0], oracle_attention_layer(c, 0))
 
 
+@pytest.mark.parametrize("Ns", [[5, 12, 9], [5, 30, 9], [5, 40, 9]], ids=["one row tile", "two row tiles", "split"])
+def test_tree_attention_long_launch_time_out_and_bad_tree_with_the_kernel_chosen_on_the_device(Ns):
+    """The same long launches as above, with the copy warps switched off (the kernel whose turn it is must
+    report the time-out and return, the others must simply leave) and with one malformed tree in the batch
+    (reported; the other sequences still match the oracle)."""
+    r = rng(8200 + Ns[1])
+    Hkv, G, n_layers = 2, 8, 26
+    Ls = [2000, 1990, 2040]
+    trees = [random_tree(r, n) for n in Ns]
+    kv = make_kv_cache(r, Ls, Ns, [l // 2 for l in Ls], Hkv, n_layers=n_layers, shuffle=True, spare_frac=0.2)
+    c = {"q": make_q(r, sum(Ns), Hkv * G, n_layers=n_layers), **kv,
+         "parent": np.concatenate([t["parent"] for t in trees]).astype(np.int32),
+         "node_offsets": np.concatenate([[0], np.cumsum(Ns)]).astype(np.int32),
+         "n_q_heads": Hkv * G, "n_kv_heads": Hkv, "head_dim": 128, "page_size": 64, "sm_scale": 0.0884}
+    st = sage.new_status()
+    sage.sage_debug_attention_waits(2_000_000, producer_off=True)
+    try:
+        gpu_attention(c, status=st)
+    finally:
+        sage.sage_debug_attention_waits(0, producer_off=False)
+    assert int(st.item()) == sage.SAGE_STATUS_TIMEOUT
+    bad = dict(c)
+    bad["parent"] = c["parent"].copy()
+    bad["parent"][Ns[0] + Ns[1] + 3] = 7                    # third tree: a parent that is not an earlier node
+    st = sage.new_status()
+    got = gpu_attention(bad, status=st)
+    assert int(st.item()) == sage.SAGE_STATUS_BAD_TREE
+    want = oracle_attention_layer(c, 1)
+    n_ok = Ns[0] + Ns[1]                                    # the first two sequences are untouched by the bad tree
+    check_attention(got[1][:n_ok], want[:n_ok])
+
+
 def test_tree_attention_is_deterministic(schedule):
     c = make_config(3, scale_down=4)
     np.testing.assert_array_equal(gpu_attention(c), gpu_attention(c))
